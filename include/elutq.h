@@ -1,0 +1,174 @@
+/*
+ * elutq.h - C ABI of the B200 (sm_100a) HLQ look-up-table GEMM/GEMV library.
+ *
+ * The library multiplies fp16 activations X[M,K] by Hierarchical-Linear-Quantized
+ * weights W_hat[N,K] without dequantising them.  HLQ (paper Section 4.1, Eq. 3)
+ * stores a weight as
+ *
+ *      W_hat[n,k] = sum_{j<q} s[n, k/G, j] * b_j[n,k] + z[n, k/G],   b_j in {0,1},
+ *
+ * with per-group, per-bit-plane fp16 scales s and per-group fp16 offsets z, groups
+ * of G consecutive k (Algorithm 1: s in R^{N x K/G x q}, z in R^{N x K/G}).  The
+ * product is evaluated with the bit-serial look-up-table procedure of Appendix B:
+ * tables of partial activation sums are built in shared memory per call, each
+ * bit-plane byte addresses a table entry, entries are summed per group in fp32,
+ * multiplied by the group's per-plane scale, and the offset contributes
+ * z[n,Gi] * sum_{k in Gi} x[k].
+ *
+ * Conventions
+ *   - All entry points return an elutq_status (0 = ok, negative = error); none
+ *     throws, aborts or traps.  Arguments are validated on the host before any
+ *     launch; on error nothing is launched and outputs are untouched.
+ *   - "device" pointers are CUDA device memory of the current device; the caller
+ *     owns every buffer it passes.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).  Work is asynchronous on `stream`.
+ *   - X, Y and `packed` must be 16-byte aligned; `planes` 8-byte aligned.
+ *   - q in [1,4]; G in {32, 64, 128}; K a multiple of G; M, N >= 1 (any value).
+ *   - Matrices are row-major and dense: X[M][K] fp16, Y[M][N] fp16 (or fp32).
+ */
+#ifndef ELUTQ_H_
+#define ELUTQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum elutq_status {
+    ELUTQ_OK = 0,
+    ELUTQ_ERR_INVALID_ARG = -1,      /* null pointer, non-positive size, bad flag combination */
+    ELUTQ_ERR_SHAPE = -2,            /* q/G out of range, K % G != 0, or (N,K) do not match the blob */
+    ELUTQ_ERR_ALIGN = -3,            /* a pointer is not aligned as required */
+    ELUTQ_ERR_BUFFER_TOO_SMALL = -4, /* packed_bytes / workspace_bytes below the required size */
+    ELUTQ_ERR_UNSUPPORTED = -5,      /* valid request this build has no kernel for */
+    ELUTQ_ERR_CUDA = -6              /* a CUDA call failed; see elutq_last_cuda_error() */
+} elutq_status;
+
+/* Flags of elutq_lut_gemm_ws / elutq_lut_gemm_f32. */
+#define ELUTQ_FLAG_SKIP_OFFSET 0x1u /* leave out the z * sum(x) term (Eq. 3 with z = 0)            */
+#define ELUTQ_FLAG_OFFSET_ONLY 0x2u /* only the z * sum(x) term; bit-planes are not read           */
+#define ELUTQ_FLAG_OUT_F32     0x4u /* Y is float[M][N] instead of fp16 (no final fp16 rounding)   */
+#define ELUTQ_FLAG_ACCUMULATE  0x8u /* Y += result (the sum is formed in fp32, rounded once)        */
+#define ELUTQ_FLAG_PLAIN_G4    0x10u /* use two 16-entry (g = 4) tables per byte instead of the
+                                        fused 256-entry table; same result up to fp32 rounding      */
+
+#define ELUTQ_HEADER_BYTES 128
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* elutq_status_string(int status);
+
+/* The cudaError_t value of the most recent failed CUDA call on this thread (0 if none). */
+int elutq_last_cuda_error(void);
+
+/*
+ * Size in bytes of the device layout of one layer (Appendix D "weight rearrange":
+ * the one-bit matrices are rearranged offline so the kernel's loads are contiguous).
+ * Pure function, no CUDA call.  The layout is q*N*K/8 bit-plane bytes +
+ * 2*(q+1)*N*K/G parameter bytes (the paper's q + 16(q+1)/G bits per weight) + a
+ * 128-byte header, with N rounded up to 16 and K to 512 by zero padding.
+ */
+int elutq_packed_bytes(int q, int G, int N, int K, size_t* bytes);
+
+/*
+ * Offline packing (Appendix B: the bit-plane split is given by the caller;
+ * Appendix D: rearrangement).  Inputs, all device memory:
+ *   planes   uint8 [q][N][K], a weight bit is (value != 0); plane j pairs with scale j
+ *   scales   fp16  [N][K/G][q]
+ *   offsets  fp16  [N][K/G]
+ * Output: `packed`, a caller-owned device buffer of at least elutq_packed_bytes()
+ * bytes, fully overwritten.  The blob is self-describing (header) and position
+ * independent: it may be copied or stored and used at another address.
+ */
+int elutq_pack(const uint8_t* planes, const void* scales, const void* offsets,
+               int q, int G, int N, int K, void* packed, size_t packed_bytes, void* stream);
+
+/*
+ * Inverse of elutq_pack (test/debug): recovers planes (uint8 0/1), scales and
+ * offsets bit-exactly into caller-owned device buffers of the shapes above.
+ */
+int elutq_unpack(const void* packed, int N, int K, uint8_t* planes, void* scales,
+                 void* offsets, void* stream);
+
+/*
+ * Reads q and G of a blob.  Blobs produced by elutq_pack in this process are
+ * known to the library; for any other device address the 128-byte header is
+ * copied to the host once (a synchronous cudaMemcpy) and remembered.
+ * Any of q, G may be NULL.  ELUTQ_ERR_SHAPE if the header is not a valid blob
+ * for (N, K).
+ */
+int elutq_describe(const void* packed, int N, int K, int* q, int* G);
+
+/* Forget what the library remembers about `packed`.  The library keys what it
+ * knows (q, G, N, K) by device address and refreshes it on elutq_pack and when
+ * (N, K) disagree; call this before freeing a blob if its address may later hold
+ * a blob of the same (N, K) but different q or G that arrives by a plain copy. */
+int elutq_forget(const void* packed);
+
+/*
+ * Scratch memory the GEMM needs for (M,N,K): per-row-block arrival counters and
+ * the fp32 partial sums of the K-split (one partial per 512-wide K chunk, summed
+ * in a fixed order by the last arriving warp, so results are bit-reproducible).
+ */
+int elutq_workspace_bytes(int M, int N, int K, size_t* bytes);
+
+/* Zero a caller-owned workspace.  Required once before its first use, and again
+ * before it is used for a different (M, N, K): the kernels leave the counters at
+ * zero after every call, but where they sit depends on the shape. */
+int elutq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Y[M,N] = X[M,K] * W_hat^T with scales and offsets applied (Eq. 3 under the
+ * bit-serial LUT procedure of Appendix B), fp32 tables and accumulation, one
+ * round-to-nearest-even conversion to fp16 at the end.
+ *   X, Y, packed: device.  Scratch comes from a library-owned per-(device,stream)
+ *   buffer that is allocated with cudaMalloc on the first call that needs it (or
+ *   needs a larger one): make one warm-up call before capturing into a CUDA graph.
+ *   Calls that share a stream are ordered; calls on different streams use
+ *   different scratch buffers.
+ */
+int elutq_lut_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
+
+/*
+ * Only the offset term of Eq. 3: Y[m,n] (+)= sum_Gi z[n,Gi] * sum_{k in Gi} X[m,k].
+ * accumulate != 0 adds into the existing fp16 Y (fp32 sum, rounded once).
+ */
+int elutq_lut_gemm_bias(const void* X, const void* packed, void* Y, int M, int N, int K,
+                        int accumulate, void* stream);
+
+/* Same product with fp32 output (no fp16 rounding) and the ELUTQ_FLAG_* options
+ * (OUT_F32 is implied).  Test/debug entry; scratch as elutq_lut_gemm. */
+int elutq_lut_gemm_f32(const void* X, const void* packed, float* Y, int M, int N, int K,
+                       unsigned flags, void* stream);
+
+/*
+ * The general entry: as above with explicit flags and a caller-owned workspace
+ * (device, 16-byte aligned, >= elutq_workspace_bytes(M,N,K), initialised by
+ * elutq_workspace_init for this shape).  Never allocates.  Two calls that run concurrently must
+ * not share a workspace.
+ */
+int elutq_lut_gemm_ws(const void* X, const void* packed, void* Y, int M, int N, int K,
+                      unsigned flags, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * End-to-end convenience for host callers: X_host (fp16 [M][K]) is copied to the
+ * device, the product runs, and Y (fp16 [M][N]) is copied back to Y_host, all on
+ * `stream` (use pinned host memory for the copies to be asynchronous).  `packed`
+ * stays a device pointer.  Staging buffers are library-owned like the scratch of
+ * elutq_lut_gemm.  The call returns without synchronising.
+ */
+int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
+                        int M, int N, int K, void* stream);
+
+/* Number of kernel launches the library has issued in this process (all entry
+ * points); lets a benchmark count its launches. */
+unsigned long long elutq_launch_count(void);
+
+/* Release every library-owned scratch/staging buffer (synchronises the device). */
+int elutq_release_scratch(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ELUTQ_H_ */

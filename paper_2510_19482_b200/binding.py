@@ -1,0 +1,164 @@
+"""ctypes binding: one Python function per C entry point, same names, argument marshalling only."""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_int, c_size_t, c_uint, c_ulonglong, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+FLAG_SKIP_OFFSET = 0x1
+FLAG_OFFSET_ONLY = 0x2
+FLAG_OUT_F32 = 0x4
+FLAG_ACCUMULATE = 0x8
+FLAG_PLAIN_G4 = 0x10
+
+
+class ElutqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().elutq_status_string(status).decode()
+        extra = f" (cudaError {lib().elutq_last_cuda_error()})" if status == -6 else ""
+        super().__init__(f"{where}: {msg}{extra} [{status}]")
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libelutq.so")
+
+
+_SIGNATURES = {
+    "elutq_status_string": (c_char_p, [c_int]),
+    "elutq_last_cuda_error": (c_int, []),
+    "elutq_packed_bytes": (c_int, [c_int, c_int, c_int, c_int, ctypes.POINTER(c_size_t)]),
+    "elutq_pack": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_size_t, c_void_p]),
+    "elutq_unpack": (c_int, [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "elutq_describe": (c_int, [c_void_p, c_int, c_int, ctypes.POINTER(c_int), ctypes.POINTER(c_int)]),
+    "elutq_forget": (c_int, [c_void_p]),
+    "elutq_workspace_bytes": (c_int, [c_int, c_int, c_int, ctypes.POINTER(c_size_t)]),
+    "elutq_workspace_init": (c_int, [c_void_p, c_size_t, c_void_p]),
+    "elutq_lut_gemm": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_lut_gemm_bias": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_void_p]),
+    "elutq_lut_gemm_f32": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p]),
+    "elutq_lut_gemm_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p, c_size_t, c_void_p]),
+    "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_launch_count": (c_ulonglong, []),
+    "elutq_release_scratch": (c_int, []),
+}
+
+
+def lib() -> ctypes.CDLL:
+    """Load libelutq.so (built in-tree by `paper_2510_19482_b200.build`); raises if it is missing."""
+    global _LIB
+    if _LIB is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise ImportError(f"{path} not found: build it with `python -m paper_2510_19482_b200.build` "
+                              "(there is no CPU fallback)")
+        handle = ctypes.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _LIB = handle
+    return _LIB
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise ElutqError(status, where)
+
+
+def _ptr(t) -> int:
+    """Raw address of a torch tensor (device or host); None -> NULL."""
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def elutq_status_string(status: int) -> str:
+    return lib().elutq_status_string(status).decode()
+
+
+def elutq_last_cuda_error() -> int:
+    return lib().elutq_last_cuda_error()
+
+
+def elutq_launch_count() -> int:
+    return int(lib().elutq_launch_count())
+
+
+def elutq_release_scratch() -> None:
+    _check(lib().elutq_release_scratch(), "elutq_release_scratch")
+
+
+def elutq_packed_bytes(q: int, G: int, N: int, K: int) -> int:
+    out = c_size_t(0)
+    _check(lib().elutq_packed_bytes(q, G, N, K, ctypes.byref(out)), "elutq_packed_bytes")
+    return out.value
+
+
+def elutq_pack(planes, scales, offsets, q: int, G: int, N: int, K: int, packed=None, stream=None):
+    """planes uint8 [q,N,K], scales fp16 [N,K/G,q], offsets fp16 [N,K/G] (CUDA tensors) -> packed uint8 blob."""
+    import torch
+    if packed is None:
+        packed = torch.empty(elutq_packed_bytes(q, G, N, K), dtype=torch.uint8, device=planes.device)
+    _check(lib().elutq_pack(_ptr(planes), _ptr(scales), _ptr(offsets), q, G, N, K,
+                            _ptr(packed), packed.numel() * packed.element_size(), _stream(stream)), "elutq_pack")
+    return packed
+
+
+def elutq_unpack(packed, N: int, K: int, planes, scales, offsets, stream=None) -> None:
+    _check(lib().elutq_unpack(_ptr(packed), N, K, _ptr(planes), _ptr(scales), _ptr(offsets), _stream(stream)),
+           "elutq_unpack")
+
+
+def elutq_describe(packed, N: int, K: int):
+    q, G = c_int(0), c_int(0)
+    _check(lib().elutq_describe(_ptr(packed), N, K, ctypes.byref(q), ctypes.byref(G)), "elutq_describe")
+    return q.value, G.value
+
+
+def elutq_forget(packed) -> None:
+    _check(lib().elutq_forget(_ptr(packed)), "elutq_forget")
+
+
+def elutq_workspace_bytes(M: int, N: int, K: int) -> int:
+    out = c_size_t(0)
+    _check(lib().elutq_workspace_bytes(M, N, K, ctypes.byref(out)), "elutq_workspace_bytes")
+    return out.value
+
+
+def elutq_workspace_init(workspace, stream=None) -> None:
+    _check(lib().elutq_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "elutq_workspace_init")
+
+
+def elutq_lut_gemm(X, packed, Y, M: int, N: int, K: int, stream=None) -> None:
+    _check(lib().elutq_lut_gemm(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, _stream(stream)), "elutq_lut_gemm")
+
+
+def elutq_lut_gemm_bias(X, packed, Y, M: int, N: int, K: int, accumulate: bool = False, stream=None) -> None:
+    _check(lib().elutq_lut_gemm_bias(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, int(bool(accumulate)), _stream(stream)),
+           "elutq_lut_gemm_bias")
+
+
+def elutq_lut_gemm_f32(X, packed, Y, M: int, N: int, K: int, flags: int = 0, stream=None) -> None:
+    _check(lib().elutq_lut_gemm_f32(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, flags, _stream(stream)),
+           "elutq_lut_gemm_f32")
+
+
+def elutq_lut_gemm_ws(X, packed, Y, M: int, N: int, K: int, flags: int, workspace, stream=None) -> None:
+    _check(lib().elutq_lut_gemm_ws(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, flags, _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream)), "elutq_lut_gemm_ws")
+
+
+def elutq_lut_gemm_host(X_host, packed, Y_host, M: int, N: int, K: int, stream=None) -> None:
+    _check(lib().elutq_lut_gemm_host(_ptr(X_host), _ptr(packed), _ptr(Y_host), M, N, K, _stream(stream)),
+           "elutq_lut_gemm_host")

@@ -1,0 +1,313 @@
+// extern "C" boundary: argument validation, blob registry, scratch management, dispatch.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <unordered_map>
+#include <utility>
+
+#include "common.cuh"
+
+namespace elutq {
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<unsigned long long> g_launches{0};
+
+struct BlobMeta { int q, G, N, K; };
+std::mutex g_mu;
+std::unordered_map<const void*, BlobMeta> g_blobs;
+
+struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
+// keyed by (device, stream, kind): kind 0 = arrival counters (always zero between calls), 1 = X staging,
+// 2 = Y staging, 3 = K-split partial sums.  Counters live in a buffer of their own so that no other data
+// is ever written where a later call with a different shape expects zeroed counters.
+std::map<std::tuple<int, void*, int>, Scratch> g_scratch;
+int g_num_sms[64] = {};
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return ELUTQ_ERR_CUDA;
+}
+
+int check_shape(int q, int G, int N, int K) {
+    if (N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    if (q < 1 || q > 4) return ELUTQ_ERR_SHAPE;
+    if (G != 32 && G != 64 && G != 128) return ELUTQ_ERR_SHAPE;
+    if (K % G != 0) return ELUTQ_ERR_SHAPE;
+    return ELUTQ_OK;
+}
+
+int num_sms() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (g_num_sms[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        g_num_sms[dev] = n;
+    }
+    return g_num_sms[dev];
+}
+
+// Workspace layout: counters (one per row block and row-batch), rounded up to 256 bytes, then partials.
+size_t counters_bytes(int M, int N) {
+    const size_t n_rb = (size_t)(N + kTileRows - 1) / kTileRows;
+    const size_t n = n_rb * (size_t)M;   // enough for any row batching of the M rows
+    return (n * sizeof(unsigned) + 255) / 256 * 256;
+}
+size_t partials_bytes(int M, int N, int K) {
+    const size_t n_rb = (size_t)(N + kTileRows - 1) / kTileRows;
+    const size_t n_kc = (size_t)(K + kChunkK - 1) / kChunkK;
+    if (n_kc <= 1) return 0;
+    return n_kc * (size_t)M * n_rb * kTileRows * sizeof(float);
+}
+
+int lookup_blob(const void* packed, int N, int K, BlobMeta* out) {
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_blobs.find(packed);
+        if (it != g_blobs.end() && it->second.N == N && it->second.K == K) {
+            *out = it->second;
+            return ELUTQ_OK;
+        }
+        // unknown address, or an entry left by a blob that has since been freed and its address
+        // reused: read the header that is there now
+    }
+    uint32_t hdr[ELUTQ_HEADER_BYTES / 4];
+    cudaError_t e = cudaMemcpy(hdr, packed, sizeof(hdr), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (hdr[0] != (uint32_t)kMagic || hdr[1] != (uint32_t)kVersion) return ELUTQ_ERR_SHAPE;
+    BlobMeta m{(int)hdr[2], (int)hdr[3], (int)hdr[4], (int)hdr[5]};
+    if (check_shape(m.q, m.G, m.N, m.K) != ELUTQ_OK || m.N != N || m.K != K) return ELUTQ_ERR_SHAPE;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_blobs[packed] = m;
+    }
+    *out = m;
+    return ELUTQ_OK;
+}
+
+// Library-owned scratch of at least `bytes` for (current device, stream, kind); counters zeroed on (re)allocation.
+int get_scratch(void* stream, int kind, size_t bytes, bool zero, void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::lock_guard<std::mutex> lk(g_mu);
+    Scratch& s = g_scratch[std::make_tuple(dev, stream, kind)];
+    if (s.bytes < bytes) {
+        if (s.ptr) {
+            e = cudaFree(s.ptr);   // synchronises: no kernel can still use the old buffer
+            s.ptr = nullptr;
+            s.bytes = 0;
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        size_t want = bytes < (1u << 20) ? (1u << 20) : bytes;
+        e = cudaMalloc(&s.ptr, want);
+        if (e != cudaSuccess) { s.ptr = nullptr; return cuda_fail(e); }
+        s.bytes = want;
+        if (zero) {
+            e = cudaMemsetAsync(s.ptr, 0, want, (cudaStream_t)stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+    }
+    *out = s.ptr;
+    return ELUTQ_OK;
+}
+
+int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, unsigned flags,
+             void* workspace, size_t workspace_bytes, bool own_workspace, void* stream) {
+    if (!X || !packed || !Y) return ELUTQ_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    if ((flags & ELUTQ_FLAG_SKIP_OFFSET) && (flags & ELUTQ_FLAG_OFFSET_ONLY)) return ELUTQ_ERR_INVALID_ARG;
+    if (flags & ~0x1fu) return ELUTQ_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(packed, 16) || !aligned(Y, 16)) return ELUTQ_ERR_ALIGN;
+    BlobMeta m;
+    int st = lookup_blob(packed, N, K, &m);
+    if (st != ELUTQ_OK) return st;
+    if ((flags & ELUTQ_FLAG_PLAIN_G4) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
+
+    const size_t cb = counters_bytes(M, N), pb = partials_bytes(M, N, K);
+    void* counters = workspace;
+    void* partials = nullptr;
+    if (own_workspace) {
+        st = get_scratch(stream, 0, cb, true, &counters);
+        if (st != ELUTQ_OK) return st;
+        st = get_scratch(stream, 3, pb ? pb : 16, false, &partials);
+        if (st != ELUTQ_OK) return st;
+    } else {
+        if (!workspace) return ELUTQ_ERR_INVALID_ARG;
+        if (!aligned(workspace, 16)) return ELUTQ_ERR_ALIGN;
+        if (workspace_bytes < cb + pb) return ELUTQ_ERR_BUFFER_TOO_SMALL;
+        partials = reinterpret_cast<uint8_t*>(workspace) + cb;
+    }
+
+    const Geo g = make_geo(m.q, m.G, N, K);
+    GemmArgs a;
+    a.X = reinterpret_cast<const __half*>(X);
+    a.tiles = reinterpret_cast<const uint8_t*>(packed) + ELUTQ_HEADER_BYTES;
+    a.Y = Y;
+    a.counters = reinterpret_cast<unsigned*>(counters);
+    a.partials = reinterpret_cast<float*>(partials);
+    a.M = M; a.N = N; a.K = K;
+    a.n_rb = g.n_rb; a.n_kc = g.n_kc;
+    a.flags = flags;
+    const int sms = num_sms();
+    int ce;
+    if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
+    else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);
+    if (ce != 0) return cuda_fail((cudaError_t)ce);
+    return ELUTQ_OK;
+}
+
+}  // namespace
+
+void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+}  // namespace elutq
+
+using namespace elutq;
+
+extern "C" {
+
+const char* elutq_status_string(int status) {
+    switch (status) {
+        case ELUTQ_OK: return "ok";
+        case ELUTQ_ERR_INVALID_ARG: return "invalid argument";
+        case ELUTQ_ERR_SHAPE: return "shape or format mismatch";
+        case ELUTQ_ERR_ALIGN: return "misaligned pointer";
+        case ELUTQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case ELUTQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ELUTQ_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+int elutq_last_cuda_error(void) { return g_last_cuda_error; }
+
+unsigned long long elutq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int elutq_packed_bytes(int q, int G, int N, int K, size_t* bytes) {
+    if (!bytes) return ELUTQ_ERR_INVALID_ARG;
+    int st = check_shape(q, G, N, K);
+    if (st != ELUTQ_OK) return st;
+    *bytes = make_geo(q, G, N, K).total_bytes;
+    return ELUTQ_OK;
+}
+
+int elutq_pack(const uint8_t* planes, const void* scales, const void* offsets, int q, int G, int N, int K,
+               void* packed, size_t packed_bytes, void* stream) {
+    if (!planes || !scales || !offsets || !packed) return ELUTQ_ERR_INVALID_ARG;
+    int st = check_shape(q, G, N, K);
+    if (st != ELUTQ_OK) return st;
+    if (!aligned(planes, 8) || !aligned(scales, 2) || !aligned(offsets, 2) || !aligned(packed, 16)) return ELUTQ_ERR_ALIGN;
+    const Geo g = make_geo(q, G, N, K);
+    if (packed_bytes < g.total_bytes) return ELUTQ_ERR_BUFFER_TOO_SMALL;
+    int ce = launch_pack(planes, reinterpret_cast<const __half*>(scales), reinterpret_cast<const __half*>(offsets), g,
+                         reinterpret_cast<uint8_t*>(packed), (cudaStream_t)stream);
+    if (ce != 0) return cuda_fail((cudaError_t)ce);
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_blobs[packed] = BlobMeta{q, G, N, K};
+    return ELUTQ_OK;
+}
+
+int elutq_unpack(const void* packed, int N, int K, uint8_t* planes, void* scales, void* offsets, void* stream) {
+    if (!packed || !planes || !scales || !offsets) return ELUTQ_ERR_INVALID_ARG;
+    if (N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(planes, 8) || !aligned(scales, 2) || !aligned(offsets, 2)) return ELUTQ_ERR_ALIGN;
+    BlobMeta m;
+    int st = lookup_blob(packed, N, K, &m);
+    if (st != ELUTQ_OK) return st;
+    const Geo g = make_geo(m.q, m.G, N, K);
+    int ce = launch_unpack(reinterpret_cast<const uint8_t*>(packed), g, planes, reinterpret_cast<__half*>(scales),
+                           reinterpret_cast<__half*>(offsets), (cudaStream_t)stream);
+    if (ce != 0) return cuda_fail((cudaError_t)ce);
+    return ELUTQ_OK;
+}
+
+int elutq_describe(const void* packed, int N, int K, int* q, int* G) {
+    if (!packed || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    BlobMeta m;
+    int st = lookup_blob(packed, N, K, &m);
+    if (st != ELUTQ_OK) return st;
+    if (q) *q = m.q;
+    if (G) *G = m.G;
+    return ELUTQ_OK;
+}
+
+int elutq_forget(const void* packed) {
+    if (!packed) return ELUTQ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_blobs.erase(packed);
+    return ELUTQ_OK;
+}
+
+int elutq_workspace_bytes(int M, int N, int K, size_t* bytes) {
+    if (!bytes || M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    *bytes = counters_bytes(M, N) + partials_bytes(M, N, K);
+    return ELUTQ_OK;
+}
+
+int elutq_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || workspace_bytes == 0) return ELUTQ_ERR_INVALID_ARG;
+    if (!aligned(workspace, 16)) return ELUTQ_ERR_ALIGN;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return ELUTQ_OK;
+}
+
+int elutq_lut_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream) {
+    return run_gemm(X, packed, Y, M, N, K, 0u, nullptr, 0, true, stream);
+}
+
+int elutq_lut_gemm_bias(const void* X, const void* packed, void* Y, int M, int N, int K, int accumulate, void* stream) {
+    const unsigned flags = ELUTQ_FLAG_OFFSET_ONLY | (accumulate ? ELUTQ_FLAG_ACCUMULATE : 0u);
+    return run_gemm(X, packed, Y, M, N, K, flags, nullptr, 0, true, stream);
+}
+
+int elutq_lut_gemm_f32(const void* X, const void* packed, float* Y, int M, int N, int K, unsigned flags, void* stream) {
+    return run_gemm(X, packed, Y, M, N, K, flags | ELUTQ_FLAG_OUT_F32, nullptr, 0, true, stream);
+}
+
+int elutq_lut_gemm_ws(const void* X, const void* packed, void* Y, int M, int N, int K, unsigned flags,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    return run_gemm(X, packed, Y, M, N, K, flags, workspace, workspace_bytes, false, stream);
+}
+
+int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host, int M, int N, int K, void* stream) {
+    if (!X_host || !packed || !Y_host) return ELUTQ_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    const size_t xb = (size_t)M * K * sizeof(__half), yb = (size_t)M * N * sizeof(__half);
+    void *xd = nullptr, *yd = nullptr;
+    int st = get_scratch(stream, 1, xb, false, &xd);
+    if (st != ELUTQ_OK) return st;
+    st = get_scratch(stream, 2, yb, false, &yd);
+    if (st != ELUTQ_OK) return st;
+    cudaError_t e = cudaMemcpyAsync(xd, X_host, xb, cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    st = run_gemm(xd, packed, yd, M, N, K, 0u, nullptr, 0, true, stream);
+    if (st != ELUTQ_OK) return st;
+    e = cudaMemcpyAsync(Y_host, yd, yb, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return ELUTQ_OK;
+}
+
+int elutq_release_scratch(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    cudaError_t first = cudaSuccess;
+    for (auto& kv : g_scratch) {
+        if (kv.second.ptr) {
+            cudaError_t e = cudaFree(kv.second.ptr);
+            if (e != cudaSuccess && first == cudaSuccess) first = e;
+        }
+    }
+    g_scratch.clear();
+    if (first != cudaSuccess) return cuda_fail(first);
+    return ELUTQ_OK;
+}
+
+}  // extern "C"

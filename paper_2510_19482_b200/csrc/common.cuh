@@ -1,0 +1,88 @@
+// Shared declarations of the CUDA side: layout geometry, launch descriptors, PTX helpers.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "elutq.h"
+
+namespace elutq {
+
+constexpr int kTileRows = 16;     // output rows per tile (one per lane of a half-warp)
+constexpr int kChunkK = 512;      // input columns per tile (64 byte-columns)
+constexpr int kMagic = 0x51544C45;
+constexpr int kVersion = 1;
+
+// Geometry of the device layout "v1" for one layer.
+//   tile = 16 rows x 512 k, stored kc-major (tile = kc * n_rb + rb).
+//   Inside a tile: plane vectors uint4 V[2q][32 lanes], then parameter words u32 P[gl*(q+1)/2][32 lanes].
+//   lane = 16*h + l: row 16*rb + l, super-groups (128 k each) h and h+2 of the chunk.
+//   Step i of a super-group visits column tau(l,i) = w*((a+v)%nsg) + (r+ii)%w,
+//   a = l/w, r = l%w, v = i/w, ii = i%w, w = G/8 columns per quantisation group, nsg = 128/G.
+struct Geo {
+    int q, G, N, K;
+    int w, nsg, gl;          // columns per group, groups per super-group, groups per lane
+    int n_rb, n_kc;
+    int tile_bytes, plane_bytes;
+    size_t total_bytes;
+};
+
+__host__ __device__ inline Geo make_geo(int q, int G, int N, int K) {
+    Geo g;
+    g.q = q; g.G = G; g.N = N; g.K = K;
+    g.w = G / 8; g.nsg = 128 / G; g.gl = 2 * g.nsg;
+    g.n_rb = (N + kTileRows - 1) / kTileRows;
+    g.n_kc = (K + kChunkK - 1) / kChunkK;
+    g.plane_bytes = 32 * 32 * q;
+    g.tile_bytes = g.plane_bytes + 32 * 2 * g.gl * (q + 1);
+    g.total_bytes = (size_t)ELUTQ_HEADER_BYTES + (size_t)g.n_kc * g.n_rb * g.tile_bytes;
+    return g;
+}
+
+// Column visited by lane-row l at step i of a super-group.
+__host__ __device__ inline int tau_of(int l, int i, int w, int nsg) {
+    const int a = l / w, r = l % w, v = i / w, ii = i % w;
+    return w * ((a + v) % nsg) + (r + ii) % w;
+}
+
+// Descriptor of one GEMM call handed to the kernel launchers.
+struct GemmArgs {
+    const __half* X;         // [M][K]
+    const uint8_t* tiles;    // packed + header
+    void* Y;                 // fp16 or fp32 [M][N]
+    float* partials;         // [n_kc][M][n_rb*16] (unused when n_kc == 1)
+    unsigned* counters;      // [n_rb * ceil(M/MB)] arrival counters, zero between calls
+    int M, N, K;
+    int n_rb, n_kc;
+    unsigned flags;
+};
+
+// Kernel launchers (defined in the .cu files); return a cudaError_t value.
+int launch_pack(const uint8_t* planes, const __half* scales, const __half* offsets,
+                const Geo& g, uint8_t* packed, cudaStream_t stream);
+int launch_unpack(const uint8_t* packed, const Geo& g, uint8_t* planes, __half* scales,
+                  __half* offsets, cudaStream_t stream);
+int launch_lut_gemv(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
+int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
+
+void count_launch(unsigned n = 1);
+
+// ---- PTX helpers -------------------------------------------------------------------------
+
+__device__ __forceinline__ uint4 ldg_stream_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ldg_stream_u32(const void* p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+// Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+}  // namespace elutq

@@ -1,0 +1,161 @@
+"""GPU parity of the M = 1 decode path against the fp64 oracle, through the C ABI.
+
+Tolerances: the kernel keeps fp32 tables and fp32 accumulators over K terms; with fp16 inputs
+the relative Frobenius error of the fp32 result is of the order sqrt(K) * 2^-24 (< 5e-6 for the
+shapes here), and the fp16 output adds one rounding of relative size <= 2^-11 per element, i.e.
+about 3e-4 in Frobenius norm.  The benchmark's bar is 1e-3 on the fp16 output.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_19482_b200 as elutq
+import workloads
+from oracle import hlq
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import gemm_f16, gemm_f32, pack_layer, x_dev  # noqa: E402
+
+TOL_F32 = 5e-6
+TOL_F16 = 1e-3
+
+# several tiles, ragged row and chunk tails, every q, every G, one-chunk (no K split) case
+SMALL = [(2, 128, 100, 1024), (3, 128, 333, 1536), (4, 128, 64, 2560), (2, 64, 50, 1088),
+         (1, 32, 17, 96), (2, 128, 16, 512), (3, 64, 1000, 4096), (4, 32, 48, 1024), (1, 128, 1, 128),
+         (2, 128, 5000, 4096)]
+
+
+def _elementwise_ok(y, ref, rel):
+    scale = np.abs(ref).max() + 1e-30
+    return np.all(np.abs(y - ref) <= rel * (np.abs(ref) + scale))
+
+
+@pytest.mark.parametrize("q,G,N,K", SMALL)
+def test_gemv_matches_oracle(q, G, N, K):
+    layer = workloads.hlq_layer(0, f"gemv/{q}/{G}/{N}/{K}", q, G, N, K, signed_scales=(q % 2 == 1))
+    X = synth.activations(0, f"gemv/x/{N}/{K}", 1, K)
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    y32 = gemm_f32(X, packed, N, K)
+    assert np.all(np.isfinite(y32))
+    assert hlq.rel_fro_error(y32, ref) <= TOL_F32
+    assert _elementwise_ok(y32, ref, 2e-5)
+    y16 = gemm_f16(X, packed, N, K)
+    assert hlq.rel_fro_error(y16, ref) <= TOL_F16
+    # the fp16 entry is the same computation with one final rounding
+    assert np.array_equal(y16.view(np.uint16), y32.astype(np.float16).view(np.uint16))
+
+
+@pytest.mark.parametrize("q,G,N,K", [(2, 128, 333, 1536), (3, 64, 50, 1088)])
+def test_offset_and_scale_terms(q, G, N, K):
+    layer = workloads.hlq_layer(1, f"terms/{q}/{G}", q, G, N, K)
+    X = synth.activations(1, "terms/x", 1, K)
+    packed = pack_layer(layer)
+    ref_scale = hlq.scale_term(X, layer.planes, layer.scales, G)
+    ref_bias = hlq.offset_term(X, layer.offsets, G)
+    y_scale = gemm_f32(X, packed, N, K, elutq.FLAG_SKIP_OFFSET)
+    y_bias = gemm_f32(X, packed, N, K, elutq.FLAG_OFFSET_ONLY)
+    y_full = gemm_f32(X, packed, N, K)
+    assert hlq.rel_fro_error(y_scale, ref_scale) <= TOL_F32
+    assert hlq.rel_fro_error(y_bias, ref_bias) <= TOL_F32
+    np.testing.assert_allclose(y_scale + y_bias, y_full, rtol=0, atol=4e-6 * np.abs(y_full).max())
+    # fp16 entry for the offset term alone, then accumulated onto the scale term
+    xd = x_dev(X)
+    Yb = torch.zeros((1, N), dtype=torch.float16, device="cuda")
+    elutq.elutq_lut_gemm_bias(xd, packed, Yb, 1, N, K, accumulate=False)
+    torch.cuda.synchronize()
+    assert hlq.rel_fro_error(Yb.cpu().numpy(), ref_bias) <= TOL_F16
+    Ya = torch.from_numpy(y_scale.astype(np.float16)).cuda()
+    elutq.elutq_lut_gemm_bias(xd, packed, Ya, 1, N, K, accumulate=True)
+    torch.cuda.synchronize()
+    assert hlq.rel_fro_error(Ya.cpu().numpy(), ref_scale + ref_bias) <= 2 * TOL_F16
+
+
+def test_f32_accumulate_flag_adds_into_y():
+    q, G, N, K = 2, 128, 100, 1024
+    layer = workloads.hlq_layer(2, "acc", q, G, N, K)
+    X = synth.activations(2, "acc/x", 1, K)
+    packed = pack_layer(layer)
+    base = gemm_f32(X, packed, N, K)
+    Y = torch.ones((1, N), dtype=torch.float32, device="cuda")
+    elutq.elutq_lut_gemm_f32(x_dev(X), packed, Y, 1, N, K, elutq.FLAG_ACCUMULATE)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(Y.cpu().numpy(), base + np.float32(1.0))
+
+
+@pytest.mark.parametrize("q", [2, 3])
+def test_plain_g4_tables_give_the_same_product(q):
+    G, N, K = 128, 333, 1536
+    layer = workloads.hlq_layer(3, f"plain/{q}", q, G, N, K)
+    X = synth.activations(3, "plain/x", 1, K)
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    y = gemm_f32(X, packed, N, K, elutq.FLAG_PLAIN_G4)
+    assert hlq.rel_fro_error(y, ref) <= TOL_F32
+
+
+def test_results_are_bit_reproducible_and_workspace_entry_agrees():
+    q, G, N, K = 3, 128, 1000, 4096
+    layer = workloads.hlq_layer(4, "repro", q, G, N, K)
+    X = synth.activations(4, "repro/x", 1, K)
+    packed = pack_layer(layer)
+    a = gemm_f16(X, packed, N, K)
+    b = gemm_f16(X, packed, N, K)
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    ws = torch.empty(elutq.elutq_workspace_bytes(1, N, K), dtype=torch.uint8, device="cuda")
+    elutq.elutq_workspace_init(ws)
+    Y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+    for _ in range(2):     # second call checks the counters returned to zero
+        Y.fill_(float("nan"))
+        elutq.elutq_lut_gemm_ws(x_dev(X), packed, Y, 1, N, K, 0, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(Y.cpu().numpy().view(np.uint16), a.view(np.uint16))
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(elutq.ElutqError) as ei:
+        elutq.elutq_lut_gemm_ws(x_dev(X), packed, Y, 1, N, K, 0, small)
+    assert ei.value.status == -4
+
+
+def test_shape_mismatch_and_degenerate_inputs():
+    q, G, N, K = 2, 128, 64, 1024
+    layer = workloads.hlq_layer(5, "degenerate", q, G, N, K)
+    packed = pack_layer(layer)
+    X = synth.activations(5, "degenerate/x", 1, K)
+    Y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+    with pytest.raises(elutq.ElutqError) as ei:
+        elutq.elutq_lut_gemm(x_dev(X), packed, Y, 1, N, K + 128)
+    assert ei.value.status == -2
+    # all-zero activations -> exactly zero; all-zero planes and scales -> offset term only
+    y0 = gemm_f32(np.zeros((1, K), np.float16), packed, N, K)
+    assert np.all(y0 == 0.0)
+    layer.planes[:] = 0
+    packed0 = pack_layer(layer)
+    ref = hlq.offset_term(X, layer.offsets, G)
+    assert hlq.rel_fro_error(gemm_f32(X, packed0, N, K), ref) <= TOL_F32
+
+
+def test_host_entry_point_round_trip():
+    q, G, N, K = 2, 128, 333, 1536
+    layer = workloads.hlq_layer(6, "host", q, G, N, K)
+    X = synth.activations(6, "host/x", 1, K)
+    packed = pack_layer(layer)
+    xh = torch.from_numpy(X.view(np.int16)).view(torch.float16).pin_memory()
+    yh = torch.empty((1, N), dtype=torch.float16).pin_memory()
+    elutq.elutq_lut_gemm_host(xh, packed, yh, 1, N, K)
+    torch.cuda.synchronize()
+    ref = gemm_f16(X, packed, N, K)
+    assert np.array_equal(yh.numpy().view(np.uint16), ref.view(np.uint16))
+
+
+def test_small_batch_rows_match_oracle():
+    # M > 1 through the same entry points (outlier activations as in the small-batch sweep)
+    q, G, N, K = 2, 128, 200, 1024
+    layer = workloads.hlq_layer(7, "batch", q, G, N, K)
+    X = synth.activations(7, "batch/x", 5, K, outliers=True)
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    assert hlq.rel_fro_error(gemm_f32(X, packed, N, K), ref) <= TOL_F32
+    assert hlq.rel_fro_error(gemm_f16(X, packed, N, K), ref) <= TOL_F16
