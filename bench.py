@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the HLQ LUT-GEMM hot path on B200.
+
+A "step" is one pass of the whole hot path (table build, weight stream, look-up/accumulate,
+per-plane scales, offset term, K-split reduce) over one batch of synthetic input: by default the
+twelve M = 1 decode linears of the LLaMA-3.1-8B shapes at q in {2,3,4}, G = 128.  One JSON line is
+printed by rank 0:
+
+  value       achieved GB/s = algorithmic bytes of the step (bit-planes + fp16 scales + fp16 offsets +
+              X + Y, summed over the calls) / device time, inputs resident in HBM, the step replayed
+              from a CUDA graph of C-ABI calls; the working set of a step exceeds the L2 capacity
+  e2e         the same metric through elutq_lut_gemm_host: X copied from pinned host memory and Y copied
+              back inside the timed region, every call
+  roofline    achieved / measured HBM copy bandwidth for the decode kernel
+  cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample of the same workload
+
+`--impl reference` times the oracle alone (the only reference there is: the paper ships no code).
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads  # noqa: E402
+from workloads import synth  # noqa: E402
+
+METRIC = "HLQ LUT-GEMM achieved HBM GB/s at M=1, 8B shapes (us/call alongside)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def _calls(name: str):
+    return {
+        "cfg0": workloads.config0,
+        "cfg1": workloads.config1_calls,
+        "cfg2": workloads.config2_calls,
+        "cfg3": workloads.config3_calls,
+        "cfg4_prefill": workloads.config4_prefill_calls,
+        "cfg4_stack": workloads.config4_stack_calls,
+    }[name]()
+
+
+WORKLOAD_NAMES = {
+    "cfg0": "config 0: single 2-bit GEMV M=1 N=K=4096 G=128",
+    "cfg1": "config 1: LLaMA-3.1-8B decode linears (qkv, o, gate_up, down) at M=1, q in {2,3,4}, G=128",
+    "cfg2": "config 2: small-batch sweep on the 8B shapes, q in {2,3}, M in {1..32}, outlier activations",
+    "cfg3": "config 3: LLaMA-3.1-70B decode linears at M=1, q in {2,3}, G=128",
+    "cfg4_prefill": "config 4a: prefill-sized GEMM on the 8B shapes, q=2, M in {128,512,2048}",
+    "cfg4_stack": "config 4b: 32-layer LLaMA-3.1-8B linear stack at M=1, q=2",
+}
+
+
+def _bytes_of(calls) -> int:
+    return sum(workloads.algorithmic_bytes(c.M, c.N, c.K, c.q, c.G) for c in calls)
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier pool measurement, MEASURED_PEAKS.json absent)"
+
+
+def _traffic_note():
+    """Per-launch DRAM traffic of the decode kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int, period_ms: int = 20):
+        self.rows = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", str(period_ms), "-i", str(device_index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.05] or [r for (_, r) in self.rows]
+        sm, smax, reasons = [], [], set()
+        for r in inside:
+            p = [x.strip() for x in r.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                sm.append(float(p[0]))
+                smax.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# ---------------------------------------------------------------------------------------------
+
+def _oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def _oracle_sample(calls, rows_per_layer: int, seed: int):
+    """Row-sampled sub-problems of the calls: (X, planes, scales, offsets, G, bytes)."""
+    out = []
+    for c in calls:
+        n = min(c.N, rows_per_layer)
+        rows = np.arange(n)
+        Gn = c.K // c.G
+        out.append((synth.activations(seed, c.tag + "/x", c.M, c.K, outliers=c.outliers),
+                    synth.bit_planes(seed, c.tag, c.q, c.N, c.K, rows=rows),
+                    synth.scales(seed, c.tag, c.N, Gn, c.q, rows=rows),
+                    synth.offsets(seed, c.tag, c.N, Gn, rows=rows),
+                    c.G, workloads.algorithmic_bytes(c.M, n, c.K, c.q, c.G)))
+    return out
+
+
+def _time_oracle(sample, steps: int, warmup: int):
+    from oracle import hlq
+    for _ in range(warmup):
+        for (X, p, s, z, G, _) in sample[:1]:
+            hlq.matmul(X, p, s, z, G)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        for (X, p, s, z, G, _) in sample:
+            hlq.matmul(X, p, s, z, G)
+    dt = (time.perf_counter() - t0) / steps
+    nbytes = sum(b for *_, b in sample)
+    return nbytes / dt / 1e9, dt
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    calls = _calls(args.workload)
+    # size the per-step sample so that steps + warmup passes of the oracle end within about two minutes
+    probe_rows = 16
+    _, probe_dt = _time_oracle(_oracle_sample(calls, probe_rows, seed=0), 1, 0)
+    budget_s = 100.0 / (args.steps + 1)
+    rows = int(max(8, min(1024, probe_rows * budget_s / max(probe_dt, 1e-6))))
+    rows -= rows % 8
+    sample = _oracle_sample(calls, rows, seed=0)
+    gbs, dt = _time_oracle(sample, args.steps, min(args.warmup, 1))
+    cores = _oracle_threads()
+    desc = f"first {rows} output rows of each of the {len(calls)} layers per step (fp64 numpy oracle)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.workload], "sample": desc},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+
+def run_cuda(args) -> None:
+    import torch
+    import torch.distributed as dist
+
+    import paper_2510_19482_b200 as elutq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+
+    calls = _calls(args.workload)
+    seed = rank           # every rank works on its own, independently drawn batch (weak scaling, no exchange)
+
+    # ---- build the workload: pack each layer once (offline step), keep X / Y per call --------------
+    layers = []
+    for c in calls:
+        lay = workloads.hlq_layer(seed, c.tag, c.q, c.G, c.N, c.K)
+        planes = torch.from_numpy(lay.planes).cuda()
+        scales = torch.from_numpy(lay.scales.view(np.int16)).cuda().view(torch.float16)
+        offsets = torch.from_numpy(lay.offsets.view(np.int16)).cuda().view(torch.float16)
+        packed = elutq.elutq_pack(planes, scales, offsets, c.q, c.G, c.N, c.K)
+        torch.cuda.synchronize()
+        del planes, scales, offsets, lay
+        Xh = torch.from_numpy(synth.activations(seed, c.tag + "/x", c.M, c.K, outliers=c.outliers).view(np.int16)) \
+            .view(torch.float16).pin_memory()
+        Yh = torch.empty((c.M, c.N), dtype=torch.float16).pin_memory()
+        layers.append(dict(call=c, packed=packed, X=Xh.cuda(), Y=torch.empty((c.M, c.N), dtype=torch.float16, device="cuda"),
+                           Xh=Xh, Yh=Yh))
+    step_bytes = _bytes_of(calls)
+    working_set = sum(l["packed"].numel() for l in layers)
+
+    def step():
+        for l in layers:
+            c = l["call"]
+            elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
+
+    def step_host():
+        for l in layers:
+            c = l["call"]
+            elutq.elutq_lut_gemm_host(l["Xh"], l["packed"], l["Yh"], c.M, c.N, c.K)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        step()              # allocates the library's scratch before capture
+        step_host()
+        stream.synchronize()
+        graph = None
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+
+        def run(n):
+            for _ in range(n):
+                if graph is not None:
+                    graph.replay()
+                else:
+                    step()
+
+        def barrier():
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        # ---- device-resident timing -------------------------------------------------------------
+        sampler = ClockSampler(local_rank) if rank == 0 else None
+        run(args.warmup)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches_before = elutq.elutq_launch_count()
+        t_wall0 = time.time()
+        e0.record()
+        run(args.steps)
+        e1.record()
+        barrier()
+        t_wall1 = time.time()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+        launches = len(calls) * args.steps if graph is not None else int(elutq.elutq_launch_count() - launches_before)
+
+        # ---- end to end through the host entry point ---------------------------------------------
+        e2e_steps = max(1, min(args.steps, 200))
+        for _ in range(min(args.warmup, 20)):
+            step_host()
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
+        for _ in range(e2e_steps):
+            step_host()
+        h1.record()
+        barrier()
+        ms_host = h0.elapsed_time(h1)
+
+        # ---- per-call times (events around single calls inside the rotating step: HBM-cold) -------
+        per_call = []
+        if rank == 0 and not args.no_per_call:
+            reps = max(3, min(args.steps, 50))
+            evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
+                   for _ in range(reps)]
+            for r in range(reps):
+                for i, l in enumerate(layers):
+                    c = l["call"]
+                    evs[r][i][0].record()
+                    elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
+                    evs[r][i][1].record()
+            torch.cuda.synchronize()
+            for i, l in enumerate(layers):
+                c = l["call"]
+                us = statistics.median(evs[r][i][0].elapsed_time(evs[r][i][1]) for r in range(reps)) * 1e3
+                b = workloads.algorithmic_bytes(c.M, c.N, c.K, c.q, c.G)
+                per_call.append({"name": c.name, "q": c.q, "M": c.M, "N": c.N, "K": c.K, "us": round(us, 3),
+                                 "GBps": round(b / us / 1e3, 1), "tflop_eq": round(2.0 * c.M * c.N * c.K / us / 1e6, 3)})
+
+    # ---- reduce over ranks ---------------------------------------------------------------------
+    t = torch.tensor([ms, ms_host], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_host = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * step_bytes / (ms_host / e2e_steps * 1e-3) / 1e9
+    peak, peak_src = _peaks()
+    per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
+    traffic = _traffic_note()
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload -------------------------
+    cpu = None
+    if not args.no_cpu_baseline:
+        rows = 1024
+        sample = _oracle_sample(calls, rows, seed=0)
+        gbs, dt = _time_oracle(sample, 1, 0)
+        cpu = {"value": gbs, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+               "sample": f"first {rows} output rows of each of the {len(calls)} layers, one pass ({dt:.1f} s)"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.workload], "calls_per_step": len(calls),
+                   "us_per_call_mean": ms_per_step * 1e3 / len(calls),
+                   "algorithmic_bytes_per_step": step_bytes, "packed_working_set_bytes": working_set,
+                   "l2": "no flush: the packed working set of a step exceeds the 126 MB L2" if working_set > 126e6
+                         else "working set fits L2 (L2-hot number, not an HBM figure)",
+                   "launch": "CUDA graph of C-ABI calls, programmatic dependent launch" if graph is not None else "stream of C-ABI calls",
+                   "parallelism": "replicas only (independent batch per rank, no collective)"},
+        "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
+                     "peak_source": peak_src,
+                     "traffic": traffic.get("dram_bytes_per_step") if traffic else None,
+                     "traffic_note": traffic.get("note") if traffic else None},
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": sum(2 * c.M * c.K for c in calls),
+                "d2h_bytes_per_step": sum(2 * c.M * c.N for c in calls)},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "cpu_baseline": cpu,
+        "per_call": per_call,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOAD_NAMES))
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-call", action="store_true")
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 2000 if args.impl == "cuda" else 10
+    if args.warmup is None:
+        args.warmup = 200 if args.impl == "cuda" else 3
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

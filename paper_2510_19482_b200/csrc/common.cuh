@@ -70,16 +70,50 @@ void count_launch(unsigned n = 1);
 
 // ---- PTX helpers -------------------------------------------------------------------------
 
+// Streaming (read-once) global loads at base + compile-time byte offset.
+template <int IMM>
 __device__ __forceinline__ uint4 ldg_stream_v4(const void* p) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "n"(IMM));
     return v;
 }
+template <int IMM>
 __device__ __forceinline__ uint32_t ldg_stream_u32(const void* p) {
     uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1+%2];" : "=r"(v) : "l"(p), "n"(IMM));
     return v;
+}
+// Compile-time loop: f(IntC<I>) for I in [0, N); IntC<I> converts to a constant int.
+template <int V>
+struct IntC {
+    static constexpr int value = V;
+    __host__ __device__ constexpr operator int() const { return V; }
+};
+template <int I, int N, class F>
+__device__ __forceinline__ void static_for(F&& f) {
+    if constexpr (I < N) {
+        f(IntC<I>{});
+        static_for<I + 1, N>(f);
+    }
+}
+// prmt.b32 in its default mode: result byte k = byte (sel nibble k & 7) of {b:a}, or that byte's
+// sign bit replicated when the nibble's bit 3 is set.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// Packed fp32x2 add (one instruction for two independent fp32 additions, round to nearest even).
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    float2 c;
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\t"
+        "mov.b64 ra, {%2, %3};\n\t"
+        "mov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rc, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}"
+        : "=f"(c.x), "=f"(c.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return c;
 }
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -20,13 +20,18 @@
 //
 // K split: one partial per K chunk goes to the workspace; the warp that arrives last at a row
 // block (arrival counter, wraps to zero) adds the partials in a fixed order and writes Y.
+#include <cstdlib>
+#include <map>
+#include <mutex>
+#include <string>
+
 #include "common.cuh"
 
 namespace elutq {
 
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kTableBytes = 256 * 256;           // 256 entries x 64 columns x 4 bytes
 constexpr int kSmemBytes = kTableBytes + 64;     // + up to 16 group sums
@@ -48,73 +53,93 @@ struct Item {
     uint32_t p[Cfg<Q, G>::NPW];
 };
 
+// vp = tile + lane*16 (plane vectors), pp = tile + PLANE_BYTES + lane*4 (parameter words);
+// every load is base + compile-time offset.
 template <int Q, int G>
-__device__ __forceinline__ void load_item(Item<Q, G>& it, const uint8_t* tile, int lane, bool planes) {
+__device__ __forceinline__ void load_item(Item<Q, G>& it, const uint8_t* vp, const uint8_t* pp, bool planes) {
     using C = Cfg<Q, G>;
-    if (planes) {
-#pragma unroll
-        for (int i = 0; i < C::NV; ++i) it.v[i] = ldg_stream_v4(tile + (i * 32 + lane) * 16);
-    }
-#pragma unroll
-    for (int i = 0; i < C::NPW; ++i) it.p[i] = ldg_stream_u32(tile + C::PLANE_BYTES + (i * 32 + lane) * 4);
+    if (planes) static_for<0, C::NV>([&](auto i) { it.v[i] = ldg_stream_v4<i * 512>(vp); });
+    static_for<0, C::NPW>([&](auto i) { it.p[i] = ldg_stream_u32<i * 128>(pp); });
 }
 
-// Builds the 64 fused tables of chunk kc and the chunk's group sums.  512 threads:
-// thread -> column c = tid & 63 and two high nibbles {2*hq, 2*hq+1}, hq = tid >> 6.
+// Builds the 64 fused tables of chunk kc and the chunk's group sums with 1024 threads.
+// lane -> column pair (2*lane, 2*lane+1); warp -> high nibble hi = warp & 15 and low-nibble half
+// lh = warp >> 4 (entries lo = 8*lh .. 8*lh+7).  Both columns are computed with packed fp32x2
+// adds and stored with one 64-bit store per entry pair (conflict-free: 256 contiguous bytes per warp).
 template <int G, bool PLAIN>
 __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __restrict__ X, int kc, int K, int tid) {
     constexpr int W = G / 8;
-    float* T = reinterpret_cast<float*>(smem);
     float* gsum = reinterpret_cast<float*>(smem + kTableBytes);
-    const int c = tid & 63, hq = tid >> 6;
-    const int k0 = kc * kChunkK + c * 8;
-    float x[8];
-    if (k0 < K) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(X + k0);
-        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+    const int lane = tid & 31, warp = tid >> 5;
+    const int hi = warp & 15, lh = warp >> 4;
+    const int k0 = kc * kChunkK + lane * 16;          // 16 activations = two byte-columns
+    float2 x[8];                                       // x[i] = (x_i of column 2*lane, x_i of column 2*lane+1)
+    if (k0 < K) {                                      // K is a multiple of 32, so both columns are in range together
+        const uint4 r0 = *reinterpret_cast<const uint4*>(X + k0);
+        const uint4 r1 = *reinterpret_cast<const uint4*>(X + k0 + 8);
+        const uint32_t a[4] = {r0.x, r0.y, r0.z, r0.w}, b[4] = {r1.x, r1.y, r1.z, r1.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
-            x[2 * i] = f.x;
-            x[2 * i + 1] = f.y;
+            const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&a[i]));
+            const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&b[i]));
+            x[2 * i] = make_float2(fa.x, fb.x);
+            x[2 * i + 1] = make_float2(fa.y, fb.y);
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = 0.f;
+        for (int i = 0; i < 8; ++i) x[i] = make_float2(0.f, 0.f);
     }
-    float A[16];
-    A[0] = 0.f;
+    // A[t] = sum of x_0..x_2 selected by the bits of t, plus x_3 for the upper half of the low nibble
+    float2 A[8];
+    A[0] = lh ? x[3] : make_float2(0.f, 0.f);
+    A[1] = fadd2(A[0], x[0]);
+    A[2] = fadd2(A[0], x[1]);
+    A[3] = fadd2(A[1], x[1]);
+    A[4] = fadd2(A[0], x[2]);
+    A[5] = fadd2(A[1], x[2]);
+    A[6] = fadd2(A[2], x[2]);
+    A[7] = fadd2(A[3], x[2]);
+    float2 Bv = make_float2(0.f, 0.f);                 // high-nibble partial sum (hi is warp-uniform)
 #pragma unroll
     for (int b = 0; b < 4; ++b)
+        if ((hi >> b) & 1) Bv = fadd2(Bv, x[4 + b]);
+    float2* row = reinterpret_cast<float2*>(smem) + (size_t)(hi * 16 + lh * 8) * 32 + lane;
+    float2 e7 = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int p = 0; p < (1 << b); ++p) A[p | (1 << b)] = A[p] + x[b];
-    float total = 0.f;
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        const int hi = 2 * hq + hh;
-        float Bv = 0.f;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) Bv += ((hi >> b) & 1) ? x[4 + b] : 0.f;
+    for (int t = 0; t < 8; ++t) {
+        float2 e;
         if (PLAIN) {
             // unfused variant: entry p holds A[lo] in rows with hi == 0 and B[hi] in rows with lo == 0
-            // (only those rows are addressed by the plain g = 4 look-ups)
-#pragma unroll
-            for (int lo = 0; lo < 16; ++lo) T[(hi * 16 + lo) * 64 + c] = (hi == 0) ? A[lo] : (lo == 0 ? Bv : 0.f);
+            const float2 zero = make_float2(0.f, 0.f);
+            e = (hi == 0) ? A[t] : ((lh == 0 && t == 0) ? Bv : zero);
         } else {
-#pragma unroll
-            for (int lo = 0; lo < 16; ++lo) T[(hi * 16 + lo) * 64 + c] = A[lo] + Bv;
+            e = fadd2(A[t], Bv);
         }
-        total = A[15] + Bv;
+        row[t * 32] = e;
+        if (t == 7) e7 = fadd2(A[t], Bv);
     }
-    if (hq == 7) {  // warps 14 and 15 hold entry 255 = sum of the column's 8 activations
+    if (warp == 31) {                                  // hi = 15, lo = 15: entry 255 = sum of the column's 8 activations
+        float total = e7.x + e7.y;
 #pragma unroll
-        for (int off = W / 2; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
-        if ((c % W) == 0) gsum[c / W] = total;
+        for (int off = W / 4; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+        if ((lane % (W / 2)) == 0) gsum[lane / (W / 2)] = total;
+    }
+}
+
+// Writes one finished output value (fp32 or fp16, optionally accumulating).
+__device__ __forceinline__ void store_out(const GemmArgs& a, int row, float y) {
+    if (a.flags & ELUTQ_FLAG_OUT_F32) {
+        float* Yf = reinterpret_cast<float*>(a.Y);
+        Yf[row] = (a.flags & ELUTQ_FLAG_ACCUMULATE) ? Yf[row] + y : y;
+    } else {
+        __half* Yh = reinterpret_cast<__half*>(a.Y);
+        if (a.flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(Yh[row]);
+        Yh[row] = __float2half_rn(y);
     }
 }
 
 template <int Q, int G, bool PLAIN>
-__global__ void __launch_bounds__(kThreads, 2) lut_gemv_kernel(const GemmArgs a) {
+__global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a) {
     using C = Cfg<Q, G>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const float* gsum = reinterpret_cast<const float*>(smem + kTableBytes);
@@ -127,14 +152,30 @@ __global__ void __launch_bounds__(kThreads, 2) lut_gemv_kernel(const GemmArgs a)
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
-    // byte offset of the lane's column inside a 256-byte table row, per step
-    uint32_t col[16];
+    // Byte offset (< 128) of the lane's column inside a 256-byte table row, per step, four steps
+    // per register: the byte-permute below picks byte (i & 3) of colp[i >> 2] as address byte 0,
+    // the weight byte as address byte 1, and zero (sign-replicated msb of a byte < 128) above.
+    uint32_t colp[4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) col[i] = 4u * (16 * h + tau_of(l, i, C::W, C::NSG));
+    for (int w4 = 0; w4 < 4; ++w4) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) v |= (4u * (16 * h + tau_of(l, 4 * w4 + b, C::W, C::NSG))) << (8 * b);
+        asm volatile("" : "+r"(v));   // keep the value in a register: recomputing it per item costs far more
+        colp[w4] = v;
+    }
 
-    Item<Q, G> cur, nxt;
+    // One register buffer per warp: every plane vector (and the parameter words) is reloaded with
+    // the next item's data right after its last use, so the loads of item i+1 are in flight while
+    // item i is processed, without a second buffer.
+    Item<Q, G> buf;
     int it = first + warp;
-    if (it < last) load_item<Q, G>(nxt, a.tiles + (size_t)it * C::TILE_BYTES, lane, use_planes);
+    // running pointers to the NEXT item to load (advance by kWarps tiles per item)
+    const uint8_t* vp = a.tiles + (size_t)it * C::TILE_BYTES + lane * 16;
+    const uint8_t* pp = a.tiles + (size_t)it * C::TILE_BYTES + C::PLANE_BYTES + lane * 4;
+    if (it < last) load_item<Q, G>(buf, vp, pp, use_planes);
+    vp += (size_t)kWarps * C::TILE_BYTES;
+    pp += (size_t)kWarps * C::TILE_BYTES;
 
     // weights do not depend on the previous kernel in the stream; X, Y and the workspace do
     grid_launch_dependents();
@@ -156,87 +197,106 @@ __global__ void __launch_bounds__(kThreads, 2) lut_gemv_kernel(const GemmArgs a)
             for (int v = 0; v < C::NSG; ++v)
                 S[u * C::NSG + v] = use_offset ? gsum[C::NSG * (h + 2 * u) + (l / C::W + v) % C::NSG] : 0.f;
 
-        while (it < seg_end) {
-            cur = nxt;
-            const int nit = it + kWarps;
-            if (nit < last) load_item<Q, G>(nxt, a.tiles + (size_t)nit * C::TILE_BYTES, lane, use_planes);
-
+        // One item: look-ups, scales, offset term, half-warp combine; with HAS_NEXT the registers of
+        // every consumed vector are refilled with the next item's data.
+        auto do_item = [&](auto has_next_c) {
+            constexpr bool HAS_NEXT = decltype(has_next_c)::value != 0;
             float prm[C::GL * (Q + 1)];
 #pragma unroll
             for (int i = 0; i < C::NPW; ++i) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&cur.p[i]));
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&buf.p[i]));
                 prm[2 * i] = f.x;
                 prm[2 * i + 1] = f.y;
             }
+            if (HAS_NEXT) static_for<0, C::NPW>([&](auto i) { buf.p[i] = ldg_stream_u32<i * 128>(pp); });
             float y = 0.f;
+            if (use_planes) {
+                static_for<0, 2 * Q>([&](auto uj) {
+                    constexpr int u = uj / Q, j = uj % Q;
+                    const uint32_t wd[4] = {buf.v[uj].x, buf.v[uj].y, buf.v[uj].z, buf.v[uj].w};
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+                    for (int v = 0; v < C::NSG; ++v) {
+                        float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int v = 0; v < C::NSG; ++v) {
-                    const int gidx = u * C::NSG + v;
-                    if (use_planes) {
+                        for (int ii = 0; ii < C::W; ii += 2) {
+                            float e[2];
 #pragma unroll
-                        for (int j = 0; j < Q; ++j) {
-                            const uint4 vec = cur.v[u * Q + j];
-                            const uint32_t wd[4] = {vec.x, vec.y, vec.z, vec.w};
-                            float acc = 0.f;
-                            if (!PLAIN) {
-#pragma unroll
-                                for (int ii = 0; ii < C::W; ++ii) {
-                                    const int i = v * C::W + ii;
-                                    const uint32_t off = __byte_perm(wd[i >> 2], col[i], 0x5504 + 0x10 * (i & 3));
-                                    acc += *reinterpret_cast<const float*>(smem + off + u * 128);
-                                }
-                            } else {
-#pragma unroll
-                                for (int ii = 0; ii < C::W; ++ii) {
-                                    const int i = v * C::W + ii;
-                                    const uint32_t off = __byte_perm(wd[i >> 2], col[i], 0x5504 + 0x10 * (i & 3));
-                                    acc += *reinterpret_cast<const float*>(smem + (off & 0x0fffu) + u * 128);   // low nibble table
-                                    acc += *reinterpret_cast<const float*>(smem + (off & 0xf0ffu) + u * 128);   // high nibble table
+                            for (int t = 0; t < 2; ++t) {
+                                const int i = v * C::W + ii + t;
+                                // address = (weight byte << 8) | lane column
+                                const uint32_t off = prmt(wd[i >> 2], colp[i >> 2], 0xCC04 + 0x11 * (i & 3));
+                                if (!PLAIN) {
+                                    e[t] = *reinterpret_cast<const float*>(smem + off + u * 128);
+                                } else {
+                                    e[t] = *reinterpret_cast<const float*>(smem + (off & 0x0fffu) + u * 128)     // low nibble table
+                                         + *reinterpret_cast<const float*>(smem + (off & 0xf0ffu) + u * 128);    // high nibble table
                                 }
                             }
-                            y = fmaf(prm[gidx * (Q + 1) + j], acc, y);
+                            acc = fadd2(acc, make_float2(e[0], e[1]));
                         }
+                        y = fmaf(prm[(u * C::NSG + v) * (Q + 1) + j], acc.x + acc.y, y);
                     }
-                    y = fmaf(prm[gidx * (Q + 1) + Q], S[gidx], y);
-                }
+                    // the vector is dead now: refill its registers with the next item's data
+                    if (HAS_NEXT) buf.v[uj] = ldg_stream_v4<uj * 512>(vp);
+                });
             }
+#pragma unroll
+            for (int gi = 0; gi < C::GL; ++gi) y = fmaf(prm[gi * (Q + 1) + Q], S[gi], y);
             y += __shfl_xor_sync(0xffffffffu, y, 16);
 
-            const int rb = it - kc * a.n_rb;
-            const int row = rb * kTileRows + l;
-            bool write_out = (a.n_kc == 1);
-            if (!write_out) {
-                if (h == 0) a.partials[(size_t)kc * n_pad + row] = y;
-                __threadfence();
-                __syncwarp();
-                unsigned old = 0;
-                if (lane == 0) old = atomicInc(a.counters + rb, (unsigned)(a.n_kc - 1));
-                old = __shfl_sync(0xffffffffu, old, 0);
-                if (old == (unsigned)(a.n_kc - 1)) {   // last chunk to arrive: fixed-order sum
-                    __threadfence();
-                    float sum = 0.f;
-                    for (int kk = h; kk < a.n_kc; kk += 2) sum += __ldcg(a.partials + (size_t)kk * n_pad + row);
-                    sum += __shfl_xor_sync(0xffffffffu, sum, 16);
-                    y = sum;
-                    write_out = true;
-                }
+            const int row = (it - kc * a.n_rb) * kTileRows + l;
+            if (a.n_kc == 1) {
+                if (h == 0 && row < a.N) store_out(a, row, y);
+            } else if (h == 0) {
+                a.partials[(size_t)kc * n_pad + row] = y;
             }
-            if (write_out && h == 0 && row < a.N) {
-                if (a.flags & ELUTQ_FLAG_OUT_F32) {
-                    float* Yf = reinterpret_cast<float*>(a.Y);
-                    Yf[row] = (a.flags & ELUTQ_FLAG_ACCUMULATE) ? Yf[row] + y : y;
-                } else {
-                    __half* Yh = reinterpret_cast<__half*>(a.Y);
-                    if (a.flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(Yh[row]);
-                    Yh[row] = __float2half_rn(y);
-                }
-            }
-            it = nit;
+        };
+
+        while (it < seg_end) {
+            if (it + kWarps < last && !(a.flags & 0x80000000u)) do_item(IntC<1>{});
+            else do_item(IntC<0>{});
+            it += kWarps;
+            vp += (size_t)kWarps * C::TILE_BYTES;
+            pp += (size_t)kWarps * C::TILE_BYTES;
         }
+
         seg = seg_end;
     }
+}
+
+// K-split epilogue: Y[n] = sum over the K chunks of partials[kc][n], chunks added in ascending order
+// (bit-reproducible), then the output conversion.  One thread per output row.  Launched right behind
+// the main kernel with programmatic dependent launch: the grid dependency wait is the only barrier.
+__global__ void __launch_bounds__(256) lut_gemv_finalize_kernel(const GemmArgs a) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= a.N) return;
+    const int n_pad = a.n_rb * kTileRows;
+    float sum = 0.f;
+    int kc = 0;
+    for (; kc + 4 <= a.n_kc; kc += 4) {
+        const float p0 = __ldcg(a.partials + (size_t)(kc + 0) * n_pad + row);
+        const float p1 = __ldcg(a.partials + (size_t)(kc + 1) * n_pad + row);
+        const float p2 = __ldcg(a.partials + (size_t)(kc + 2) * n_pad + row);
+        const float p3 = __ldcg(a.partials + (size_t)(kc + 3) * n_pad + row);
+        sum = (((sum + p0) + p1) + p2) + p3;
+    }
+    for (; kc < a.n_kc; ++kc) sum += __ldcg(a.partials + (size_t)kc * n_pad + row);
+    store_out(a, row, sum);
+}
+
+// Debug switches read once from the environment (0 when unset): launch-shape experiments only.
+inline int debug_env(const char* name) {
+    static std::map<std::string, int> cache;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(name);
+    if (it != cache.end()) return it->second;
+    const char* v = getenv(name);
+    const int val = v ? atoi(v) : 0;
+    cache[name] = val;
+    return val;
 }
 
 template <int Q, int G, bool PLAIN>
@@ -251,8 +311,9 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     }
     const long long total = (long long)a.n_kc * a.n_rb;
     if (total >= (1LL << 31) - kWarps) return (int)cudaErrorInvalidValue;
-    long long grid = (total + kWarps - 1) / kWarps;
-    if (grid > num_sms) grid = 2LL * num_sms;
+    long long grid = (total + kWarps - 1) / kWarps;      // at least one item per warp where possible
+    if (grid > num_sms) grid = num_sms;                   // one 1024-thread CTA per SM
+    if (debug_env("ELUTQ_DEBUG_GRID") > 0) grid = debug_env("ELUTQ_DEBUG_GRID");
     if (grid > total) grid = total;
     if (grid < 1) grid = 1;
 
@@ -265,8 +326,17 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, a);
+    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
+    GemmArgs b = a;
+    if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;   // timing experiment: skip reloads (results invalid)
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
+    count_launch(1);
+    if (e != cudaSuccess || a.n_kc == 1) return (int)e;
+    cudaLaunchConfig_t fcfg = cfg;
+    fcfg.gridDim = dim3((unsigned)((a.N + 255) / 256));
+    fcfg.blockDim = dim3(256);
+    fcfg.dynamicSmemBytes = 0;
+    e = cudaLaunchKernelEx(&fcfg, lut_gemv_finalize_kernel, b);
     count_launch(1);
     return (int)e;
 }
