@@ -56,6 +56,7 @@ struct GemmArgs {
     int M, N, K;
     int n_rb, n_kc;
     unsigned flags;
+    int items_q, items_r;    // items per CTA: CTA b owns items_q (+1 if b < items_r) consecutive items
 };
 
 // Kernel launchers (defined in the .cu files); return a cudaError_t value.

@@ -146,23 +146,26 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
-    const long long total = (long long)a.n_kc * a.n_rb;   // < 2^31 (checked by the launcher)
-    const int first = (int)(total * blockIdx.x / gridDim.x);
-    const int last = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    const int bid = blockIdx.x;
+    const int first = bid * a.items_q + min(bid, a.items_r);
+    const int last = first + a.items_q + (bid < a.items_r ? 1 : 0);
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
     // Byte offset (< 128) of the lane's column inside a 256-byte table row, per step, four steps
     // per register: the byte-permute below picks byte (i & 3) of colp[i >> 2] as address byte 0,
     // the weight byte as address byte 1, and zero (sign-replicated msb of a byte < 128) above.
+    // Four steps share a phase (W >= 4), so the four bytes are computed at once:
+    // tau = W*((a+v) % NSG) + (r + ii0 + b) % W for b = 0..3.
     uint32_t colp[4];
 #pragma unroll
     for (int w4 = 0; w4 < 4; ++w4) {
-        uint32_t v = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) v |= (4u * (16 * h + tau_of(l, 4 * w4 + b, C::W, C::NSG))) << (8 * b);
-        asm volatile("" : "+r"(v));   // keep the value in a register: recomputing it per item costs far more
-        colp[w4] = v;
+        const int v = (4 * w4) / C::W, ii0 = (4 * w4) % C::W;
+        const uint32_t base = 16u * h + C::W * (((l / C::W) + v) % C::NSG);
+        const uint32_t t = (((uint32_t)(l % C::W) + ii0) * 0x01010101u + 0x03020100u) & ((C::W - 1) * 0x01010101u);
+        uint32_t vcol = (t + base * 0x01010101u) << 2;
+        asm volatile("" : "+r"(vcol));   // keep the value in a register: recomputing it per item costs far more
+        colp[w4] = vcol;
     }
 
     // One register buffer per warp: every plane vector (and the parameter words) is reloaded with
@@ -328,6 +331,8 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     cfg.attrs = attr;
     cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
     GemmArgs b = a;
+    b.items_q = (int)(total / grid);
+    b.items_r = (int)(total % grid);
     if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;   // timing experiment: skip reloads (results invalid)
     cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
     count_launch(1);
