@@ -161,6 +161,25 @@ int elutq_lut_gemm_ws(const void* X, const void* packed, void* Y, int M, int N, 
 int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
                         int M, int N, int K, void* stream);
 
+/*
+ * (No counterpart in the paper: an addition for deployments that must not allocate.)
+ * Same product as elutq_lut_gemm - Y[M,N] fp16 = X[M,K] * W_hat^T, all device pointers - for
+ * callers that cannot allocate device memory: a component embedded in a runtime that owns the
+ * whole device arena, a decode loop that cannot afford the device-wide stall of cudaMalloc or
+ * cudaFree, a process held to a fixed memory budget.  The K-split scratch lives in a 4 MiB array
+ * that is part of the library image on every GPU that loads it; the call never invokes
+ * cudaMalloc, cudaFree or any allocating routine.
+ *   - Limit: ceil(K/512) * M * 16*ceil(N/16) * 4 bytes must not exceed 4 MiB (every M = 1
+ *     LLaMA-3.1 8B/70B shape fits); larger requests return ELUTQ_ERR_BUFFER_TOO_SMALL and
+ *     launch nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the array, which keeps the previous call's contents (nothing
+ *     needs clearing: every value read was written by the same call).  Calls that overlap on the
+ *     GPU, e.g. on different streams, race on it: keep them stream-ordered.
+ */
+int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
+
 /* Number of kernel launches the library has issued in this process (all entry
  * points); lets a benchmark count its launches. */
 unsigned long long elutq_launch_count(void);

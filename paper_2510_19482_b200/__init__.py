@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     elutq_lut_gemm_f32,
     elutq_lut_gemm_ws,
     elutq_lut_gemm_host,
+    elutq_lut_gemm_static,
     elutq_launch_count,
     elutq_release_scratch,
     elutq_status_string,

@@ -43,6 +43,7 @@ _SIGNATURES = {
     "elutq_lut_gemm_f32": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p]),
     "elutq_lut_gemm_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p, c_size_t, c_void_p]),
     "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_lut_gemm_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
 }
@@ -162,3 +163,9 @@ def elutq_lut_gemm_ws(X, packed, Y, M: int, N: int, K: int, flags: int, workspac
 def elutq_lut_gemm_host(X_host, packed, Y_host, M: int, N: int, K: int, stream=None) -> None:
     _check(lib().elutq_lut_gemm_host(_ptr(X_host), _ptr(packed), _ptr(Y_host), M, N, K, _stream(stream)),
            "elutq_lut_gemm_host")
+
+
+def elutq_lut_gemm_static(X, packed, Y, M: int, N: int, K: int, stream=None) -> None:
+    """elutq_lut_gemm for callers that must not allocate: scratch is a fixed 4 MiB array inside the library."""
+    _check(lib().elutq_lut_gemm_static(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, _stream(stream)),
+           "elutq_lut_gemm_static")

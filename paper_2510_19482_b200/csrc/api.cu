@@ -168,6 +168,18 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
 
 void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Helpers for entry points that live in other translation units.
+int blob_meta(const void* packed, int N, int K, int* q, int* G) {
+    BlobMeta m;
+    const int st = lookup_blob(packed, N, K, &m);
+    if (st != ELUTQ_OK) return st;
+    *q = m.q;
+    *G = m.G;
+    return ELUTQ_OK;
+}
+int note_cuda_error(int cuda_error) { return cuda_fail((cudaError_t)cuda_error); }
+int device_sm_count() { return num_sms(); }
+
 }  // namespace elutq
 
 using namespace elutq;

@@ -69,6 +69,12 @@ int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t s
 
 void count_launch(unsigned n = 1);
 
+// api.cu helpers shared with other translation units: blob description (registry or header read),
+// recording a CUDA error for elutq_last_cuda_error(), SM count of the current device.
+int blob_meta(const void* packed, int N, int K, int* q, int* G);
+int note_cuda_error(int cuda_error);
+int device_sm_count();
+
 // ---- PTX helpers -------------------------------------------------------------------------
 
 // Streaming (read-once) global loads at base + compile-time byte offset.

@@ -1,0 +1,56 @@
+"""elutq_lut_gemm_static: the entry point for callers that cannot allocate device memory.
+
+Collected last on purpose (file name), so a run that stops at the first failure has already run
+every other test.  The entry point keeps its K-split scratch in a fixed array inside the library,
+so it must give the same result as elutq_lut_gemm, call after call, with no set-up by the caller.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_19482_b200 as elutq
+import workloads
+from oracle import hlq
+from workloads import synth
+
+TOL_F16 = 1e-3
+
+
+def test_static_entry_rejects_shapes_beyond_its_scratch_before_any_launch():
+    # 16 chunks * 64 rows * 57344 output rows * 4 bytes is far above the 4 MiB built-in scratch
+    L = elutq.lib()
+    before = elutq.elutq_launch_count()
+    assert L.elutq_lut_gemm_static(16, 16, 16, 64, 57344, 8192, None) == -4
+    assert L.elutq_lut_gemm_static(None, 16, 16, 1, 64, 1024, None) == -1
+    assert L.elutq_lut_gemm_static(8, 16, 16, 1, 64, 1024, None) == -3
+    assert elutq.elutq_launch_count() == before
+
+
+@pytest.mark.gpu
+def test_static_entry_matches_the_allocating_entry_on_two_calls_in_a_row():
+    from gpu_util import pack_layer, x_dev
+
+    q, G, N, K = 3, 128, 1000, 4096            # 8-way K split, ragged row tail
+    layer = workloads.hlq_layer(11, "static", q, G, N, K)
+    packed = pack_layer(layer)
+    ref64 = None
+    for call in range(2):                       # second call reuses the array with the first call's leftovers in it
+        X = synth.activations(11 + call, "static/x", 1, K)
+        xd = x_dev(X)
+        Y_ref = torch.empty((1, N), dtype=torch.float16, device="cuda")
+        elutq.elutq_lut_gemm(xd, packed, Y_ref, 1, N, K)
+        Y = torch.full((1, N), float("nan"), dtype=torch.float16, device="cuda")
+        elutq.elutq_lut_gemm_static(xd, packed, Y, 1, N, K)
+        torch.cuda.synchronize()
+        got, want = Y.cpu().numpy(), Y_ref.cpu().numpy()
+        assert np.all(np.isfinite(got))
+        assert hlq.rel_fro_error(got, want) <= TOL_F16
+        ref64 = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+        assert hlq.rel_fro_error(got, ref64) <= TOL_F16
+    # a small batch goes through the same entry
+    Xb = synth.activations(13, "static/xb", 3, K)
+    Yb = torch.empty((3, N), dtype=torch.float16, device="cuda")
+    elutq.elutq_lut_gemm_static(x_dev(Xb), packed, Yb, 3, N, K)
+    torch.cuda.synchronize()
+    assert hlq.rel_fro_error(Yb.cpu().numpy(), hlq.matmul(Xb, layer.planes, layer.scales, layer.offsets, G)) <= TOL_F16
