@@ -107,9 +107,10 @@ int elutq_describe(const void* packed, int N, int K, int* q, int* G);
 int elutq_forget(const void* packed);
 
 /*
- * Scratch memory the GEMM needs for (M,N,K): per-row-block arrival counters and
- * the fp32 partial sums of the K-split (one partial per 512-wide K chunk, summed
- * in a fixed order by the last arriving warp, so results are bit-reproducible).
+ * Scratch memory the GEMM needs for (M,N,K): a small reserved control area and the
+ * fp32 partial sums of the K-split (one partial per 512-wide K chunk for M = 1, per
+ * 256-wide half chunk for M > 1, summed in ascending chunk order by the finalize
+ * kernel, so results are bit-reproducible).
  */
 int elutq_workspace_bytes(int M, int N, int K, size_t* bytes);
 
@@ -169,9 +170,9 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
  * cudaFree, a process held to a fixed memory budget.  The K-split scratch lives in a 4 MiB array
  * that is part of the library image on every GPU that loads it; the call never invokes
  * cudaMalloc, cudaFree or any allocating routine.
- *   - Limit: ceil(K/512) * M * 16*ceil(N/16) * 4 bytes must not exceed 4 MiB (every M = 1
- *     LLaMA-3.1 8B/70B shape fits); larger requests return ELUTQ_ERR_BUFFER_TOO_SMALL and
- *     launch nothing.
+ *   - Limit: C * M * 16*ceil(N/16) * 4 bytes must not exceed 4 MiB, with C = ceil(K/512) K
+ *     chunks for M = 1 and C = 2*ceil(K/512) for M > 1 (every M = 1 LLaMA-3.1 8B/70B shape
+ *     fits); larger requests return ELUTQ_ERR_BUFFER_TOO_SMALL and launch nothing.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call before any stream capture begins.
  *   - All calls on a device share the array, which keeps the previous call's contents (nothing

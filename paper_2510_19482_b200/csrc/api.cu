@@ -63,8 +63,10 @@ size_t counters_bytes(int M, int N) {
 size_t partials_bytes(int M, int N, int K) {
     const size_t n_rb = (size_t)(N + kTileRows - 1) / kTileRows;
     const size_t n_kc = (size_t)(K + kChunkK - 1) / kChunkK;
-    if (n_kc <= 1) return 0;
-    return n_kc * (size_t)M * n_rb * kTileRows * sizeof(float);
+    // M = 1: one partial per 512-column chunk (none when there is a single chunk);
+    // M > 1: one per 256-column half chunk
+    const size_t chunks = (M == 1) ? (n_kc > 1 ? n_kc : 0) : 2 * n_kc;
+    return chunks * (size_t)M * n_rb * kTileRows * sizeof(float);
 }
 
 int lookup_blob(const void* packed, int N, int K, BlobMeta* out) {

@@ -67,6 +67,8 @@ int launch_unpack(const uint8_t* packed, const Geo& g, uint8_t* planes, __half* 
 int launch_lut_gemv(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 
+int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream);
+int debug_env(const char* name);
 void count_launch(unsigned n = 1);
 
 // api.cu helpers shared with other translation units: blob description (registry or header read),
@@ -121,6 +123,17 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
         "mov.b64 {%0, %1}, rc;\n\t}"
         : "=f"(c.x), "=f"(c.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
     return c;
+}
+// Writes one finished output value Y[idx] (fp32 or fp16, optionally accumulating).
+__device__ __forceinline__ void store_out(const GemmArgs& a, size_t idx, float y) {
+    if (a.flags & ELUTQ_FLAG_OUT_F32) {
+        float* Yf = reinterpret_cast<float*>(a.Y);
+        Yf[idx] = (a.flags & ELUTQ_FLAG_ACCUMULATE) ? Yf[idx] + y : y;
+    } else {
+        __half* Yh = reinterpret_cast<__half*>(a.Y);
+        if (a.flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(Yh[idx]);
+        Yh[idx] = __float2half_rn(y);
+    }
 }
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

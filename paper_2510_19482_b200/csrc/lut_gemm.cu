@@ -1,20 +1,311 @@
-// M > 1: small-batch / prefill LUT GEMM.
+// M > 1: small-batch / prefill LUT GEMM over the same packed layout.
+//
+// MB activation rows (2 or 4) are processed per pass: a table entry holds the partial sums of all MB
+// rows for one (byte value, column), so one weight byte costs one byte-permute, one 8- or 16-byte
+// shared-memory load and MB/2 packed fp32x2 adds.  Tables of one pass cover half a tile (256 input
+// columns = super-groups 2u and 2u+1 of a chunk): 256 entries x 32 columns x MB floats.
+//
+// Work list: (row batch mb, half chunk kc2 = 2*kc + u, row block rb), flattened in that order and cut
+// into equal contiguous ranges, one per CTA (one 1024-thread CTA per SM); tables are rebuilt when a
+// range crosses an (mb, kc2) boundary.  Partial sums go to partials[kc2][m][n]; the finalize kernel adds
+// the 2*n_kc half chunks in ascending order.  The look-up rate of shared memory (one 4-byte entry per
+// lane per cycle per SM), not HBM, bounds this path: time grows with M.
 #include "common.cuh"
 
 namespace elutq {
 
-int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream) {
-    // Row-at-a-time: every activation row runs the decode kernel (correct for any M).
-    const size_t ybytes = (a.flags & ELUTQ_FLAG_OUT_F32) ? sizeof(float) : sizeof(__half);
-    for (int m = 0; m < a.M; ++m) {
-        GemmArgs r = a;
-        r.M = 1;
-        r.X = a.X + (size_t)m * a.K;
-        r.Y = reinterpret_cast<uint8_t*>(a.Y) + (size_t)m * a.N * ybytes;
-        int e = launch_lut_gemv(r, q, G, num_sms, stream);
-        if (e != 0) return e;
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kHalfK = 256;                        // input columns covered by one table set
+
+template <int Q, int G, int MB>
+struct BCfg {
+    static constexpr int W = G / 8;
+    static constexpr int NSG = 128 / G;
+    static constexpr int NPW = 2 * NSG * (Q + 1) / 2;          // parameter words per lane (both halves)
+    static constexpr int PLANE_BYTES = 1024 * Q;
+    static constexpr int TILE_BYTES = PLANE_BYTES + 128 * NPW;
+    static constexpr int ENTRY_BYTES = 4 * MB;                 // one table entry: MB floats
+    static constexpr int TABLE_BYTES = 256 * 32 * ENTRY_BYTES; // 64 KiB (MB = 2) or 128 KiB (MB = 4)
+    static constexpr int SMEM_BYTES = TABLE_BYTES + (256 / G) * MB * 4 + 64;
+};
+
+// Tables of half chunk kc2 for rows m0 .. m0+MB-1: lane -> column c (8 activations of every row),
+// warp -> high nibble hi = warp & 15 and low-nibble half lh = warp >> 4.  Rows are paired in the
+// packed adds.  Rows >= M and columns >= K contribute zeros.
+template <int G, int MB>
+__device__ __forceinline__ void build_tables_mb(uint8_t* smem, int table_bytes, const __half* __restrict__ X,
+                                                int M, int K, int m0, int kc2, int tid) {
+    constexpr int W = G / 8;
+    constexpr int NP = MB / 2;                          // row pairs
+    float* gsum = reinterpret_cast<float*>(smem + table_bytes);   // [256/G groups][MB]
+    const int lane = tid & 31, warp = tid >> 5;
+    const int hi = warp & 15, lh = warp >> 4;
+    const int k0 = kc2 * kHalfK + lane * 8;
+    float2 x[NP][8];                                    // x[p][i] = (x_i of row m0+2p, x_i of row m0+2p+1)
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        float xa[8], xb[8];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int m = m0 + 2 * p + r;
+            float* dst = r ? xb : xa;
+            if (m < M && k0 < K) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                    dst[2 * i] = f.x;
+                    dst[2 * i + 1] = f.y;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) dst[i] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
     }
-    return 0;
+    float2 e7[NP];
+    uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * (4 * MB) + lane * (4 * MB);
+    float2 A[NP][8], Bv[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
+        A[p][1] = fadd2(A[p][0], x[p][0]);
+        A[p][2] = fadd2(A[p][0], x[p][1]);
+        A[p][3] = fadd2(A[p][1], x[p][1]);
+        A[p][4] = fadd2(A[p][0], x[p][2]);
+        A[p][5] = fadd2(A[p][1], x[p][2]);
+        A[p][6] = fadd2(A[p][2], x[p][2]);
+        A[p][7] = fadd2(A[p][3], x[p][2]);
+        Bv[p] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        float2 e[NP];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) e[p] = fadd2(A[p][t], Bv[p]);
+        uint8_t* dst = rowp + (size_t)t * 32 * (4 * MB);
+        if (MB == 2) *reinterpret_cast<float2*>(dst) = e[0];
+        else *reinterpret_cast<float4*>(dst) = make_float4(e[0].x, e[0].y, e[NP - 1].x, e[NP - 1].y);
+        if (t == 7) {
+#pragma unroll
+            for (int p = 0; p < NP; ++p) e7[p] = e[p];
+        }
+    }
+    if (warp == 31) {   // entry 255: the column's activation sums; reduce over the W columns of a group
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            float sx = e7[p].x, sy = e7[p].y;
+#pragma unroll
+            for (int off = W / 2; off >= 1; off >>= 1) {
+                sx += __shfl_xor_sync(0xffffffffu, sx, off);
+                sy += __shfl_xor_sync(0xffffffffu, sy, off);
+            }
+            if ((lane % W) == 0) {
+                gsum[(lane / W) * MB + 2 * p] = sx;
+                gsum[(lane / W) * MB + 2 * p + 1] = sy;
+            }
+        }
+    }
+}
+
+template <int Q, int G, int MB>
+__global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a) {
+    using C = BCfg<Q, G, MB>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const float* gsum = reinterpret_cast<const float*>(smem + C::TABLE_BYTES);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int h = lane >> 4, l = lane & 15;
+    const int bid = blockIdx.x;
+    const int first = bid * a.items_q + min(bid, a.items_r);
+    const int last = first + a.items_q + (bid < a.items_r ? 1 : 0);
+    const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
+    const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
+    const int n_kc2 = 2 * a.n_kc;
+    const int per_mb = n_kc2 * a.n_rb;                 // items per row batch
+    const size_t n_pad = (size_t)a.n_rb * kTileRows;
+
+    // Lane column byte offsets inside a table row (column * 8 bytes; the address is doubled for MB = 4),
+    // three steps per register, the fourth byte stays zero and supplies the upper address bytes.
+    uint32_t colp[6];
+#pragma unroll
+    for (int w3 = 0; w3 < 6; ++w3) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int b = 0; b < 3; ++b) {
+            const int i = 3 * w3 + b;
+            if (i < 16) v |= (8u * (16 * h + tau_of(l, i, C::W, C::NSG))) << (8 * b);
+        }
+        asm volatile("" : "+r"(v));
+        colp[w3] = v;
+    }
+
+    grid_launch_dependents();
+    grid_dependency_wait();
+
+    int seg = first;
+    while (seg < last) {
+        const int mb = seg / per_mb;
+        const int rem = seg - mb * per_mb;
+        const int kc2 = rem / a.n_rb;
+        const int seg_end = min(last, mb * per_mb + (kc2 + 1) * a.n_rb);
+        const int m0 = mb * MB;
+        const int u = kc2 & 1;
+        __syncthreads();
+        build_tables_mb<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
+        __syncthreads();
+
+        // group sums of this lane's groups in this half: group (NSG*h + (a+v) % NSG) of the half
+        float S[C::NSG][MB];
+#pragma unroll
+        for (int v = 0; v < C::NSG; ++v)
+#pragma unroll
+            for (int m = 0; m < MB; ++m)
+                S[v][m] = use_offset ? gsum[(C::NSG * h + (l / C::W + v) % C::NSG) * MB + m] : 0.f;
+
+        for (int it = seg + warp; it < seg_end; it += kWarps) {
+            const int rb = it - mb * per_mb - kc2 * a.n_rb;
+            const uint8_t* tile = a.tiles + ((size_t)(kc2 >> 1) * a.n_rb + rb) * C::TILE_BYTES;
+            uint4 vec[Q];
+            uint32_t pw[C::NPW];
+            if (use_planes) static_for<0, Q>([&](auto j) { vec[j] = ldg_stream_v4<0>(tile + ((u * Q + j) * 32 + lane) * 16); });
+            static_for<0, C::NPW>([&](auto i) { pw[i] = ldg_stream_u32<0>(tile + C::PLANE_BYTES + (i * 32 + lane) * 4); });
+            float prm_all[2 * C::NPW];
+#pragma unroll
+            for (int i = 0; i < C::NPW; ++i) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&pw[i]));
+                prm_all[2 * i] = f.x;
+                prm_all[2 * i + 1] = f.y;
+            }
+            float prm[C::NSG * (Q + 1)];               // this half's records (static indexing keeps it in registers)
+#pragma unroll
+            for (int i = 0; i < C::NSG * (Q + 1); ++i) prm[i] = u ? prm_all[C::NSG * (Q + 1) + i] : prm_all[i];
+            float y[MB];
+#pragma unroll
+            for (int m = 0; m < MB; ++m) y[m] = 0.f;
+            if (use_planes) {
+#pragma unroll
+                for (int j = 0; j < Q; ++j) {
+                    const uint32_t wd[4] = {vec[j].x, vec[j].y, vec[j].z, vec[j].w};
+#pragma unroll
+                    for (int v = 0; v < C::NSG; ++v) {
+                        float2 acc[MB / 2];
+#pragma unroll
+                        for (int p = 0; p < MB / 2; ++p) acc[p] = make_float2(0.f, 0.f);
+#pragma unroll
+                        for (int ii = 0; ii < C::W; ++ii) {
+                            const int i = v * C::W + ii;
+                            // address byte 0 = lane column, byte 1 = weight byte, bytes 2..3 = 0
+                            const uint32_t off = prmt(wd[i >> 2], colp[i / 3], 0x7704 + 0x10 * (i & 3) + (i % 3));
+                            if (MB == 2) {
+                                const float2 e = *reinterpret_cast<const float2*>(smem + off);
+                                acc[0] = fadd2(acc[0], e);
+                            } else {
+                                const float4 e = *reinterpret_cast<const float4*>(smem + 2 * off);
+                                acc[0] = fadd2(acc[0], make_float2(e.x, e.y));
+                                acc[MB / 2 - 1] = fadd2(acc[MB / 2 - 1], make_float2(e.z, e.w));
+                            }
+                        }
+                        const float s = prm[v * (Q + 1) + j];
+#pragma unroll
+                        for (int p = 0; p < MB / 2; ++p) {
+                            y[2 * p] = fmaf(s, acc[p].x, y[2 * p]);
+                            y[2 * p + 1] = fmaf(s, acc[p].y, y[2 * p + 1]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int v = 0; v < C::NSG; ++v) {
+                const float z = prm[v * (Q + 1) + Q];
+#pragma unroll
+                for (int m = 0; m < MB; ++m) y[m] = fmaf(z, S[v][m], y[m]);
+            }
+#pragma unroll
+            for (int m = 0; m < MB; ++m) y[m] += __shfl_xor_sync(0xffffffffu, y[m], 16);
+            if (h == 0) {
+                const int row = rb * kTileRows + l;
+#pragma unroll
+                for (int m = 0; m < MB; ++m)
+                    if (m0 + m < a.M) a.partials[((size_t)kc2 * a.M + (m0 + m)) * n_pad + row] = y[m];
+            }
+        }
+        seg = seg_end;
+    }
+}
+
+template <int Q, int G, int MB>
+int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
+    using C = BCfg<Q, G, MB>;
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(lut_gemm_kernel<Q, G, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e != cudaSuccess) return (int)e;
+        configured[dev] = true;
+    }
+    const int n_mb = (a.M + MB - 1) / MB;
+    const long long total = (long long)n_mb * 2 * a.n_kc * a.n_rb;
+    if (total >= (1LL << 31) - kWarps) return (int)cudaErrorInvalidValue;
+    long long grid = (total + kWarps - 1) / kWarps;
+    if (grid > num_sms) grid = num_sms;
+    if (grid < 1) grid = 1;
+    GemmArgs b = a;
+    b.items_q = (int)(total / grid);
+    b.items_r = (int)(total % grid);
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB>, b);
+    count_launch(1);
+    if (e != cudaSuccess) return (int)e;
+    return launch_finalize(b, 2 * a.n_kc, cfg.numAttrs != 0, stream);
+}
+
+template <int Q, int G>
+int launch_qg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
+    return a.M == 2 ? launch_mb<Q, G, 2>(a, num_sms, stream) : launch_mb<Q, G, 4>(a, num_sms, stream);
+}
+
+template <int Q>
+int launch_q(const GemmArgs& a, int G, int num_sms, cudaStream_t stream) {
+    switch (G) {
+        case 32: return launch_qg<Q, 32>(a, num_sms, stream);
+        case 64: return launch_qg<Q, 64>(a, num_sms, stream);
+        case 128: return launch_qg<Q, 128>(a, num_sms, stream);
+        default: return (int)cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream) {
+    if (a.flags & ELUTQ_FLAG_PLAIN_G4) return (int)cudaErrorNotSupported;   // decode-kernel variant only
+    switch (q) {
+        case 1: return launch_q<1>(a, G, num_sms, stream);
+        case 2: return launch_q<2>(a, G, num_sms, stream);
+        case 3: return launch_q<3>(a, G, num_sms, stream);
+        case 4: return launch_q<4>(a, G, num_sms, stream);
+        default: return (int)cudaErrorInvalidValue;
+    }
 }
 
 }  // namespace elutq

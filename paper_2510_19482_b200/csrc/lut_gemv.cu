@@ -126,18 +126,6 @@ __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __rest
     }
 }
 
-// Writes one finished output value (fp32 or fp16, optionally accumulating).
-__device__ __forceinline__ void store_out(const GemmArgs& a, int row, float y) {
-    if (a.flags & ELUTQ_FLAG_OUT_F32) {
-        float* Yf = reinterpret_cast<float*>(a.Y);
-        Yf[row] = (a.flags & ELUTQ_FLAG_ACCUMULATE) ? Yf[row] + y : y;
-    } else {
-        __half* Yh = reinterpret_cast<__half*>(a.Y);
-        if (a.flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(Yh[row]);
-        Yh[row] = __float2half_rn(y);
-    }
-}
-
 template <int Q, int G, bool PLAIN>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a) {
     using C = Cfg<Q, G>;
@@ -249,7 +237,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
 
             const int row = (it - kc * a.n_rb) * kTileRows + l;
             if (a.n_kc == 1) {
-                if (h == 0 && row < a.N) store_out(a, row, y);
+                if (h == 0 && row < a.N) store_out(a, (size_t)row, y);
             } else if (h == 0) {
                 a.partials[(size_t)kc * n_pad + row] = y;
             }
@@ -267,30 +255,35 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     }
 }
 
-// K-split epilogue: Y[n] = sum over the K chunks of partials[kc][n], chunks added in ascending order
-// (bit-reproducible), then the output conversion.  One thread per output row.  Launched right behind
-// the main kernel with programmatic dependent launch: the grid dependency wait is the only barrier.
-__global__ void __launch_bounds__(256) lut_gemv_finalize_kernel(const GemmArgs a) {
+// K-split epilogue: Y[m][n] = sum over the K chunks of partials[chunk][m][n], chunks added in ascending
+// order (bit-reproducible), then the output conversion.  One thread per output element.  Launched right
+// behind the main kernel with programmatic dependent launch: the grid dependency wait is the only barrier.
+__global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, const int n_chunks) {
     grid_launch_dependents();
     grid_dependency_wait();
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= a.N) return;
-    const int n_pad = a.n_rb * kTileRows;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)a.M * a.N) return;
+    const int m = (int)(idx / a.N), row = (int)(idx % a.N);
+    const size_t n_pad = (size_t)a.n_rb * kTileRows;
+    const float* p = a.partials + (size_t)m * n_pad + row;
+    const size_t stride = (size_t)a.M * n_pad;
     float sum = 0.f;
-    int kc = 0;
-    for (; kc + 4 <= a.n_kc; kc += 4) {
-        const float p0 = __ldcg(a.partials + (size_t)(kc + 0) * n_pad + row);
-        const float p1 = __ldcg(a.partials + (size_t)(kc + 1) * n_pad + row);
-        const float p2 = __ldcg(a.partials + (size_t)(kc + 2) * n_pad + row);
-        const float p3 = __ldcg(a.partials + (size_t)(kc + 3) * n_pad + row);
+    int c = 0;
+    for (; c + 4 <= n_chunks; c += 4) {
+        const float p0 = __ldcg(p + (size_t)(c + 0) * stride);
+        const float p1 = __ldcg(p + (size_t)(c + 1) * stride);
+        const float p2 = __ldcg(p + (size_t)(c + 2) * stride);
+        const float p3 = __ldcg(p + (size_t)(c + 3) * stride);
         sum = (((sum + p0) + p1) + p2) + p3;
     }
-    for (; kc < a.n_kc; ++kc) sum += __ldcg(a.partials + (size_t)kc * n_pad + row);
-    store_out(a, row, sum);
+    for (; c < n_chunks; ++c) sum += __ldcg(p + (size_t)c * stride);
+    store_out(a, (size_t)m * a.N + row, sum);
 }
 
+}  // namespace
+
 // Debug switches read once from the environment (0 when unset): launch-shape experiments only.
-inline int debug_env(const char* name) {
+int debug_env(const char* name) {
     static std::map<std::string, int> cache;
     static std::mutex mu;
     std::lock_guard<std::mutex> lk(mu);
@@ -301,6 +294,23 @@ inline int debug_env(const char* name) {
     cache[name] = val;
     return val;
 }
+
+int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(((long long)a.M * a.N + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_finalize_kernel, a, n_chunks);
+    count_launch(1);
+    return (int)e;
+}
+
+namespace {
 
 template <int Q, int G, bool PLAIN>
 int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
@@ -337,13 +347,7 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
     count_launch(1);
     if (e != cudaSuccess || a.n_kc == 1) return (int)e;
-    cudaLaunchConfig_t fcfg = cfg;
-    fcfg.gridDim = dim3((unsigned)((a.N + 255) / 256));
-    fcfg.blockDim = dim3(256);
-    fcfg.dynamicSmemBytes = 0;
-    e = cudaLaunchKernelEx(&fcfg, lut_gemv_finalize_kernel, b);
-    count_launch(1);
-    return (int)e;
+    return launch_finalize(b, a.n_kc, cfg.numAttrs != 0, stream);
 }
 
 template <int Q>

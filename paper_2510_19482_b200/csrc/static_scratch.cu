@@ -54,10 +54,12 @@ extern "C" int elutq_lut_gemm_static(const void* X, const void* packed, void* Y,
     if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(packed) || !aligned16(Y)) return ELUTQ_ERR_ALIGN;
 
-    // K-split partial sums: one fp32 per (K chunk, activation row, padded output row)
+    // K-split partial sums: one fp32 per (K chunk, activation row, padded output row); chunks are
+    // 512 columns wide for M = 1 and 256 columns wide for M > 1
     const size_t n_rb = ((size_t)N + kTileRows - 1) / kTileRows;
     const size_t n_kc = ((size_t)K + kChunkK - 1) / kChunkK;
-    const size_t need = n_kc > 1 ? n_kc * (size_t)M * n_rb * kTileRows * sizeof(float) : 0;
+    const size_t chunks = (M == 1) ? (n_kc > 1 ? n_kc : 0) : 2 * n_kc;
+    const size_t need = chunks * (size_t)M * n_rb * kTileRows * sizeof(float);
     if (need > ELUTQ_STATIC_SCRATCH_BYTES) return ELUTQ_ERR_BUFFER_TOO_SMALL;   // shape exceeds the built-in scratch
 
     int q = 0, G = 0;
