@@ -211,6 +211,21 @@ def run_reference(args) -> None:
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 
+def max_over_ranks(values_ms, device="cuda"):
+    """Element-wise maximum of per-rank timings over all ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values_ms), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(step_bytes: int, world: int, ms_per_step: float) -> float:
+    """Whole-job GB/s: every rank processes its own batch of step_bytes in the (max-over-ranks) step time."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+
 def run_cuda(args) -> None:
     import torch
     import torch.distributed as dist
@@ -310,39 +325,58 @@ def run_cuda(args) -> None:
         barrier()
         ms_host = h0.elapsed_time(h1)
 
-        # ---- per-call times (events around single calls inside the rotating step: HBM-cold) -------
+        # ---- per-call times: marginal device time of one extra call inside the graph-replayed step -------
+        # (the extra call reads its own copy of the packed layer, so it is HBM-cold like the others and
+        #  does not warm the L2 for the step's own call)
         per_call = []
-        if rank == 0 and not args.no_per_call:
-            reps = max(3, min(args.steps, 50))
-            evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
-                   for _ in range(reps)]
-            for r in range(reps):
-                for i, l in enumerate(layers):
-                    c = l["call"]
-                    evs[r][i][0].record()
-                    elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
-                    evs[r][i][1].record()
-            torch.cuda.synchronize()
-            for i, l in enumerate(layers):
+        if rank == 0 and not args.no_per_call and graph is not None:
+            reps = max(20, min(args.steps, 300))
+
+            def time_graph(g):
+                for _ in range(3):
+                    g.replay()
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a0.record()
+                for _ in range(reps):
+                    g.replay()
+                a1.record()
+                torch.cuda.synchronize()
+                return a0.elapsed_time(a1) * 1e3 / reps
+
+            seen = {}
+            for l in layers:
                 c = l["call"]
-                us = statistics.median(evs[r][i][0].elapsed_time(evs[r][i][1]) for r in range(reps)) * 1e3
+                key = (c.name.split(".")[-1], c.q, c.M, c.N, c.K)
+                if key in seen:
+                    continue
+                seen[key] = True
+                clone = l["packed"].clone()
+                elutq.elutq_describe(clone, c.N, c.K)
+                Y2 = torch.empty_like(l["Y"])
+                g2 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g2, stream=stream):
+                    elutq.elutq_lut_gemm(l["X"], clone, Y2, c.M, c.N, c.K)
+                    step()
+                t_base = time_graph(graph)
+                us = max(time_graph(g2) - t_base, 0.0)
                 b = workloads.algorithmic_bytes(c.M, c.N, c.K, c.q, c.G)
-                per_call.append({"name": c.name, "q": c.q, "M": c.M, "N": c.N, "K": c.K, "us": round(us, 3),
-                                 "GBps": round(b / us / 1e3, 1), "tflop_eq": round(2.0 * c.M * c.N * c.K / us / 1e6, 3)})
+                per_call.append({"name": key[0], "q": c.q, "M": c.M, "N": c.N, "K": c.K, "us": round(us, 3),
+                                 "GBps": round(b / max(us, 1e-3) / 1e3, 1),
+                                 "frac_of_hbm_peak": round(b / max(us, 1e-3) / 1e3 / _peaks()[0], 3),
+                                 "tflop_eq": round(2.0 * c.M * c.N * c.K / max(us, 1e-3) / 1e6, 3)})
+                elutq.elutq_forget(clone)
+                del g2, clone, Y2
 
     # ---- reduce over ranks ---------------------------------------------------------------------
-    t = torch.tensor([ms, ms_host], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_host = float(t[0]), float(t[1])
+    ms, ms_host = max_over_ranks([ms, ms_host])
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     ms_per_step = ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * step_bytes / (ms_host / e2e_steps * 1e-3) / 1e9
+    value = aggregate_value(step_bytes, world, ms_per_step)
+    e2e_value = aggregate_value(step_bytes, world, ms_host / e2e_steps)
     peak, peak_src = _peaks()
     per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
     traffic = _traffic_note()
