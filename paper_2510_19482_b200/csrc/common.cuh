@@ -57,6 +57,11 @@ struct GemmArgs {
     int n_rb, n_kc;
     unsigned flags;
     int items_q, items_r;    // items per CTA: CTA b owns items_q (+1 if b < items_r) consecutive items
+    int active_warps;        // warps that take items (item stride); the rest only help build tables
+    int ranges, rb_q, rb_r;  // aligned partition: every chunk is cut into the same `ranges` row ranges (0 = flat
+                             // partition of the item list); range r holds rb_q (+1 if r < rb_r) row blocks;
+                             // CTA b = chunk * ranges + r
+    int fused_reduce;        // 1: the last CTA of a range reduces it in-kernel (needs counters); 0: finalize kernel
 };
 
 // Kernel launchers (defined in the .cu files); return a cudaError_t value.

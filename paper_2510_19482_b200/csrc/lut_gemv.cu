@@ -34,7 +34,7 @@ namespace {
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kTableBytes = 256 * 256;           // 256 entries x 64 columns x 4 bytes
-constexpr int kSmemBytes = kTableBytes + 64;     // + up to 16 group sums
+constexpr int kSmemBytes = kTableBytes + 128;    // + up to 16 group sums + the reduction flag
 
 template <int Q, int G>
 struct Cfg {
@@ -126,6 +126,39 @@ __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __rest
     }
 }
 
+// Sum of n partial sums p[0], p[stride], ... in ascending order (the order fixes the rounding, so the
+// result is bit-reproducible); loads are issued 16 at a time so that a reduction costs one or two
+// L2 round trips instead of one per chunk.
+__device__ __forceinline__ float sum_chunks(const float* p, size_t stride, int n) {
+    float sum = 0.f;
+    int c = 0;
+    for (; c + 16 <= n; c += 16) {
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __ldcg(p + (size_t)(c + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum += v[i];
+    }
+    if (c + 8 <= n) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __ldcg(p + (size_t)(c + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += v[i];
+        c += 8;
+    }
+    if (c + 4 <= n) {
+        float v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = __ldcg(p + (size_t)(c + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sum += v[i];
+        c += 4;
+    }
+    for (; c < n; ++c) sum += __ldcg(p + (size_t)c * stride);
+    return sum;
+}
+
 template <int Q, int G, bool PLAIN>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a) {
     using C = Cfg<Q, G>;
@@ -135,8 +168,20 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
     const int bid = blockIdx.x;
-    const int first = bid * a.items_q + min(bid, a.items_r);
-    const int last = first + a.items_q + (bid < a.items_r ? 1 : 0);
+    int first, last, range = 0, range_rb0 = 0, range_rb1 = 0;
+    if (a.ranges > 0) {
+        // aligned partition: every chunk is cut into the same `ranges` row ranges, so the chunks of one
+        // range can be reduced by whichever of their CTAs finishes last
+        const int kc_own = bid / a.ranges;
+        range = bid - kc_own * a.ranges;
+        range_rb0 = range * a.rb_q + min(range, a.rb_r);
+        range_rb1 = range_rb0 + a.rb_q + (range < a.rb_r ? 1 : 0);
+        first = kc_own * a.n_rb + range_rb0;
+        last = kc_own * a.n_rb + range_rb1;
+    } else {
+        first = bid * a.items_q + min(bid, a.items_r);
+        last = first + a.items_q + (bid < a.items_r ? 1 : 0);
+    }
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
@@ -160,13 +205,14 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     // the next item's data right after its last use, so the loads of item i+1 are in flight while
     // item i is processed, without a second buffer.
     Item<Q, G> buf;
-    int it = first + warp;
+    const int stride = a.active_warps;
+    int it = warp < stride ? first + warp : last;
     // running pointers to the NEXT item to load (advance by kWarps tiles per item)
     const uint8_t* vp = a.tiles + (size_t)it * C::TILE_BYTES + lane * 16;
     const uint8_t* pp = a.tiles + (size_t)it * C::TILE_BYTES + C::PLANE_BYTES + lane * 4;
     if (it < last) load_item<Q, G>(buf, vp, pp, use_planes);
-    vp += (size_t)kWarps * C::TILE_BYTES;
-    pp += (size_t)kWarps * C::TILE_BYTES;
+    vp += (size_t)stride * C::TILE_BYTES;
+    pp += (size_t)stride * C::TILE_BYTES;
 
     // weights do not depend on the previous kernel in the stream; X, Y and the workspace do
     grid_launch_dependents();
@@ -244,14 +290,36 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         };
 
         while (it < seg_end) {
-            if (it + kWarps < last && !(a.flags & 0x80000000u)) do_item(IntC<1>{});
+            if (it + stride < last && !(a.flags & 0x80000000u)) do_item(IntC<1>{});
             else do_item(IntC<0>{});
-            it += kWarps;
-            vp += (size_t)kWarps * C::TILE_BYTES;
-            pp += (size_t)kWarps * C::TILE_BYTES;
+            it += stride;
+            vp += (size_t)stride * C::TILE_BYTES;
+            pp += (size_t)stride * C::TILE_BYTES;
         }
 
         seg = seg_end;
+    }
+
+    if (a.fused_reduce && a.n_kc > 1) {
+        // In-kernel K-split reduction: each CTA publishes its partials and takes one ticket for its row
+        // range; the CTA that draws the last ticket of the range adds the chunks in ascending order
+        // (bit-reproducible) and writes Y.  The counter wraps to zero, ready for the next call.
+        int* flag = reinterpret_cast<int*>(smem + kTableBytes + 64);
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const unsigned old = atomicInc(a.counters + range, (unsigned)(a.n_kc - 1));
+            *flag = (old == (unsigned)(a.n_kc - 1)) ? 1 : 0;
+        }
+        __syncthreads();
+        if (*flag) {
+            __threadfence();
+            const int row_end = min(range_rb1 * kTileRows, a.N);
+            for (int row = range_rb0 * kTileRows + tid; row < row_end; row += kThreads) {
+                const float* p = a.partials + row;
+                store_out(a, (size_t)row, sum_chunks(p, (size_t)n_pad, a.n_kc));
+            }
+        }
     }
 }
 
@@ -267,17 +335,7 @@ __global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, con
     const size_t n_pad = (size_t)a.n_rb * kTileRows;
     const float* p = a.partials + (size_t)m * n_pad + row;
     const size_t stride = (size_t)a.M * n_pad;
-    float sum = 0.f;
-    int c = 0;
-    for (; c + 4 <= n_chunks; c += 4) {
-        const float p0 = __ldcg(p + (size_t)(c + 0) * stride);
-        const float p1 = __ldcg(p + (size_t)(c + 1) * stride);
-        const float p2 = __ldcg(p + (size_t)(c + 2) * stride);
-        const float p3 = __ldcg(p + (size_t)(c + 3) * stride);
-        sum = (((sum + p0) + p1) + p2) + p3;
-    }
-    for (; c < n_chunks; ++c) sum += __ldcg(p + (size_t)c * stride);
-    store_out(a, (size_t)m * a.N + row, sum);
+    store_out(a, (size_t)m * a.N + row, sum_chunks(p, stride, n_chunks));
 }
 
 }  // namespace
@@ -343,10 +401,34 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     GemmArgs b = a;
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
+    // Aligned partition (one table build per CTA, no chunk crossings) when it keeps >= 90 % of the SMs busy
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0;
+    if (a.n_kc > 1 && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
+        int R = num_sms / a.n_kc;
+        const int r_cap = (a.n_rb + kWarps - 1) / kWarps;   // keep at least one item per warp (fewer CTAs = fewer table builds)
+        if (R > r_cap) R = r_cap;
+        if (R >= 1 && (long long)R * a.n_kc * 10 >= 9LL * (grid < num_sms ? grid : num_sms)) {
+            b.ranges = R;
+            b.rb_q = a.n_rb / R;
+            b.rb_r = a.n_rb % R;
+            grid = (long long)R * a.n_kc;
+            cfg.gridDim = dim3((unsigned)grid);
+            b.fused_reduce = (a.counters != nullptr && debug_env("ELUTQ_DEBUG_FUSED") > 0) ? 1 : 0;
+        }
+    }
+    {   // even rounds: with R = ceil(items/32) rounds, ceil(items/R) warps take items
+        const int items_max = b.items_q + (b.items_r ? 1 : 0);
+        const int rounds = (items_max + kWarps - 1) / kWarps;
+        b.active_warps = kWarps;   // measured: evening out the rounds (ceil(items/rounds) warps) gains nothing
+        (void)rounds;
+        if (debug_env("ELUTQ_DEBUG_WARPS") > 0) b.active_warps = debug_env("ELUTQ_DEBUG_WARPS");
+        if (b.active_warps > kWarps) b.active_warps = kWarps;
+        if (b.active_warps < 1) b.active_warps = 1;
+    }
     if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;   // timing experiment: skip reloads (results invalid)
     cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
     count_launch(1);
-    if (e != cudaSuccess || a.n_kc == 1) return (int)e;
+    if (e != cudaSuccess || a.n_kc == 1 || b.fused_reduce) return (int)e;
     return launch_finalize(b, a.n_kc, cfg.numAttrs != 0, stream);
 }
 
