@@ -43,6 +43,13 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 def _calls(name: str):
+    if name.startswith("custom:"):
+        # custom:q:N:K[:M],q:N:K[:M],...  (G = 128) - used for profiler captures of single shapes
+        out = []
+        for i, spec in enumerate(name[len("custom:"):].split(",")):
+            f = [int(x) for x in spec.split(":")]
+            out.append(workloads.shapes.Call(f"custom{i}", f[3] if len(f) > 3 else 1, f[1], f[2], f[0]))
+        return out
     return {
         "cfg0": workloads.config0,
         "cfg1": workloads.config1_calls,
@@ -424,11 +431,16 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOAD_NAMES))
+    ap.add_argument("--workload", default="cfg1",
+                    help="one of %s, or custom:q:N:K[:M],... (G = 128)" % ", ".join(sorted(WORKLOAD_NAMES)))
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-call", action="store_true")
     args = ap.parse_args()
+    if args.workload not in WORKLOAD_NAMES:
+        if not args.workload.startswith("custom:"):
+            ap.error("unknown workload")
+        WORKLOAD_NAMES[args.workload] = "custom shapes " + args.workload[len("custom:"):]
     if args.steps is None:
         args.steps = 2000 if args.impl == "cuda" else 10
     if args.warmup is None:

@@ -14,6 +14,7 @@ from .synth import (  # noqa: F401
     offsets,
     outlier_columns,
 )
+from . import shapes  # noqa: F401
 from .shapes import (  # noqa: F401
     LLAMA31_8B,
     LLAMA31_70B,
