@@ -60,7 +60,8 @@ struct GemmArgs {
     int active_warps;        // warps that take items (item stride); the rest only help build tables
     int ranges, rb_q, rb_r;  // aligned partition: every chunk is cut into the same `ranges` row ranges (0 = flat
                              // partition of the item list); range r holds rb_q (+1 if r < rb_r) row blocks;
-                             // CTA b = chunk * ranges + r
+                             // CTA b = group * ranges + r, group = `cpc` consecutive chunks
+    int cpc;                 // chunks per CTA in the aligned partition
     int fused_reduce;        // 1: the last CTA of a range reduces it in-kernel (needs counters); 0: finalize kernel
 };
 

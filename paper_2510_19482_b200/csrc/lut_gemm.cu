@@ -264,7 +264,7 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
     b.active_warps = kWarps;
-    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0;
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

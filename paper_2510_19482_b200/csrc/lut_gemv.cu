@@ -168,16 +168,21 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
     const int bid = blockIdx.x;
-    int first, last, range = 0, range_rb0 = 0, range_rb1 = 0;
+    // Work of this CTA: `nseg` segments of consecutive items; segment s starts at first + s * (len + jump).
+    //   aligned partition: one segment per chunk of the CTA's chunk group, all over the same row range
+    //                      (so one table build per chunk and no CTA straddles a chunk boundary)
+    //   flat partition:    one contiguous range of the kc-major item list (jump = 0), cut at chunk ends
+    int first, last, jump = 0, range = 0, range_rb0 = 0, range_rb1 = 0;
     if (a.ranges > 0) {
-        // aligned partition: every chunk is cut into the same `ranges` row ranges, so the chunks of one
-        // range can be reduced by whichever of their CTAs finishes last
-        const int kc_own = bid / a.ranges;
-        range = bid - kc_own * a.ranges;
+        const int grp = bid / a.ranges;
+        range = bid - grp * a.ranges;
         range_rb0 = range * a.rb_q + min(range, a.rb_r);
         range_rb1 = range_rb0 + a.rb_q + (range < a.rb_r ? 1 : 0);
-        first = kc_own * a.n_rb + range_rb0;
-        last = kc_own * a.n_rb + range_rb1;
+        const int kc0 = grp * a.cpc;
+        const int nseg = min(a.cpc, a.n_kc - kc0);
+        first = kc0 * a.n_rb + range_rb0;
+        last = (kc0 + nseg - 1) * a.n_rb + range_rb1;       // end of the last segment
+        jump = a.n_rb - (range_rb1 - range_rb0);
     } else {
         first = bid * a.items_q + min(bid, a.items_r);
         last = first + a.items_q + (bid < a.items_r ? 1 : 0);
@@ -206,13 +211,17 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     // item i is processed, without a second buffer.
     Item<Q, G> buf;
     const int stride = a.active_warps;
-    int it = warp < stride ? first + warp : last;
-    // running pointers to the NEXT item to load (advance by kWarps tiles per item)
-    const uint8_t* vp = a.tiles + (size_t)it * C::TILE_BYTES + lane * 16;
-    const uint8_t* pp = a.tiles + (size_t)it * C::TILE_BYTES + C::PLANE_BYTES + lane * 4;
-    if (it < last) load_item<Q, G>(buf, vp, pp, use_planes);
-    vp += (size_t)stride * C::TILE_BYTES;
-    pp += (size_t)stride * C::TILE_BYTES;
+    const int seg_len0 = (a.ranges > 0) ? (range_rb1 - range_rb0) : (last - first);
+    // first item of this warp: position `warp` in the concatenated segments
+    int it = last, it_end = first + seg_len0;                // it_end: end of the segment `it` lies in
+    if (warp < stride) {
+        it = first + warp;
+        while (it >= it_end && it_end < last) { it += jump; it_end += a.n_rb; }
+        if (it >= it_end) it = last;
+    }
+    if (it < last)
+        load_item<Q, G>(buf, a.tiles + (size_t)it * C::TILE_BYTES + lane * 16,
+                        a.tiles + (size_t)it * C::TILE_BYTES + C::PLANE_BYTES + lane * 4, use_planes);
 
     // weights do not depend on the previous kernel in the stream; X, Y and the workspace do
     grid_launch_dependents();
@@ -222,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     int seg = first;
     while (seg < last) {
         const int kc = seg / a.n_rb;
-        const int seg_end = min(last, (kc + 1) * a.n_rb);
+        const int seg_end = (a.ranges > 0) ? seg + seg_len0 : min(last, (kc + 1) * a.n_rb);
         __syncthreads();
         build_tables<G, PLAIN>(smem, a.X, kc, a.K, tid);
         __syncthreads();
@@ -234,6 +243,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
             for (int v = 0; v < C::NSG; ++v)
                 S[u * C::NSG + v] = use_offset ? gsum[C::NSG * (h + 2 * u) + (l / C::W + v) % C::NSG] : 0.f;
 
+        const uint8_t* nvp = nullptr;     // next item's plane vectors / parameter words for this lane
+        const uint8_t* npp = nullptr;
         // One item: look-ups, scales, offset term, half-warp combine; with HAS_NEXT the registers of
         // every consumed vector are refilled with the next item's data.
         auto do_item = [&](auto has_next_c) {
@@ -245,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
                 prm[2 * i] = f.x;
                 prm[2 * i + 1] = f.y;
             }
-            if (HAS_NEXT) static_for<0, C::NPW>([&](auto i) { buf.p[i] = ldg_stream_u32<i * 128>(pp); });
+            if (HAS_NEXT) static_for<0, C::NPW>([&](auto i) { buf.p[i] = ldg_stream_u32<i * 128>(npp); });
             float y = 0.f;
             if (use_planes) {
                 static_for<0, 2 * Q>([&](auto uj) {
@@ -274,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
                         y = fmaf(prm[(u * C::NSG + v) * (Q + 1) + j], acc.x + acc.y, y);
                     }
                     // the vector is dead now: refill its registers with the next item's data
-                    if (HAS_NEXT) buf.v[uj] = ldg_stream_v4<uj * 512>(vp);
+                    if (HAS_NEXT) buf.v[uj] = ldg_stream_v4<uj * 512>(nvp);
                 });
             }
 #pragma unroll
@@ -290,14 +301,19 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         };
 
         while (it < seg_end) {
-            if (it + stride < last && !(a.flags & 0x80000000u)) do_item(IntC<1>{});
+            // next item of this warp: `stride` positions further in the concatenated segments
+            int nit = it + stride, nend = it_end;
+            while (nit >= nend && nend < last) { nit += jump; nend += a.n_rb; }
+            const bool has_next = nit < nend && !(a.flags & 0x80000000u);
+            nvp = a.tiles + (size_t)nit * C::TILE_BYTES + lane * 16;
+            npp = nvp + (C::PLANE_BYTES - lane * 12);
+            if (has_next) do_item(IntC<1>{});
             else do_item(IntC<0>{});
-            it += stride;
-            vp += (size_t)stride * C::TILE_BYTES;
-            pp += (size_t)stride * C::TILE_BYTES;
+            it = (nit < nend) ? nit : last;
+            it_end = nend;
         }
 
-        seg = seg_end;
+        seg = (a.ranges > 0) ? seg + a.n_rb : seg_end;
     }
 
     if (a.fused_reduce && a.n_kc > 1) {
@@ -333,9 +349,7 @@ __global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, con
     if (idx >= (long long)a.M * a.N) return;
     const int m = (int)(idx / a.N), row = (int)(idx % a.N);
     const size_t n_pad = (size_t)a.n_rb * kTileRows;
-    const float* p = a.partials + (size_t)m * n_pad + row;
-    const size_t stride = (size_t)a.M * n_pad;
-    store_out(a, (size_t)m * a.N + row, sum_chunks(p, stride, n_chunks));
+    store_out(a, (size_t)m * a.N + row, sum_chunks(a.partials + (size_t)m * n_pad + row, (size_t)a.M * n_pad, n_chunks));
 }
 
 }  // namespace
@@ -355,6 +369,7 @@ int debug_env(const char* name) {
 
 int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
+    // one thread per output element: the reduction is latency-bound, so it wants all the parallelism it can get
     cfg.gridDim = dim3((unsigned)(((long long)a.M * a.N + 255) / 256));
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
@@ -382,8 +397,7 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     }
     const long long total = (long long)a.n_kc * a.n_rb;
     if (total >= (1LL << 31) - kWarps) return (int)cudaErrorInvalidValue;
-    long long grid = (total + kWarps - 1) / kWarps;      // at least one item per warp where possible
-    if (grid > num_sms) grid = num_sms;                   // one 1024-thread CTA per SM
+    long long grid = total < num_sms ? total : num_sms;   // one 1024-thread CTA per SM
     if (debug_env("ELUTQ_DEBUG_GRID") > 0) grid = debug_env("ELUTQ_DEBUG_GRID");
     if (grid > total) grid = total;
     if (grid < 1) grid = 1;
@@ -401,19 +415,43 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     GemmArgs b = a;
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
-    // Aligned partition (one table build per CTA, no chunk crossings) when it keeps >= 90 % of the SMs busy
-    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0;
+    // Aligned partition: groups of `cpc` consecutive chunks x R row ranges, one CTA each.  Pick the cpc
+    // that keeps the SMs busiest (work / (SMs * largest CTA share)); fall back to the flat partition
+    // of the item list when no choice reaches 80 %.
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1;
     if (a.n_kc > 1 && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
-        int R = num_sms / a.n_kc;
-        const int r_cap = (a.n_rb + kWarps - 1) / kWarps;   // keep at least one item per warp (fewer CTAs = fewer table builds)
-        if (R > r_cap) R = r_cap;
-        if (R >= 1 && (long long)R * a.n_kc * 10 >= 9LL * (grid < num_sms ? grid : num_sms)) {
-            b.ranges = R;
-            b.rb_q = a.n_rb / R;
-            b.rb_r = a.n_rb % R;
-            grid = (long long)R * a.n_kc;
+        // Cost model in item times: the kernel lasts as long as its largest CTA, i.e. that CTA's items
+        // plus ~16 item times per table build (measured: an extra build costs far more than the
+        // imbalance it could remove).  Minimise that makespan over the aligned choices and the flat one.
+        const double kBuild = 16.0;
+        const long long flat_grid = total < num_sms ? total : num_sms;
+        const long long flat_items = (total + flat_grid - 1) / flat_grid;
+        double best = (double)flat_items + kBuild * (double)((flat_items + a.n_rb - 1) / a.n_rb + 1);   // flat partition
+        int best_cpc = 0, best_R = 0;
+        const int force_cpc = debug_env("ELUTQ_DEBUG_CPC"), force_R = debug_env("ELUTQ_DEBUG_R");
+        for (int cpc = 1; cpc <= 8 && cpc <= a.n_kc; ++cpc) {
+            if (force_cpc > 0 && cpc != force_cpc) continue;
+            const int groups = (a.n_kc + cpc - 1) / cpc;
+            int R = num_sms / groups;
+            // Short kernels (< ~100 items per CTA) run faster in a stream of calls when about 20 SMs stay
+            // free for the early-launched CTAs of the kernels that follow (measured: 128 CTAs beat 144 by
+            // ~12 % on 20-25 MB layers); long kernels want every SM.
+            const int R_spare = (num_sms - 20) / groups;
+            if (R_spare >= 1 && (a.n_rb + R - 1) / R < 100) R = R_spare;
+            if (R > a.n_rb) R = a.n_rb;
+            if (force_R > 0 && force_R < R) R = force_R;
+            if (R < 1) continue;
+            const double span = (double)cpc * ((double)((a.n_rb + R - 1) / R) + kBuild);
+            if (span < best - 1e-9 || force_cpc > 0) { best = span; best_cpc = cpc; best_R = R; }
+        }
+        if (best_cpc > 0) {
+            b.cpc = best_cpc;
+            b.ranges = best_R;
+            b.rb_q = a.n_rb / best_R;
+            b.rb_r = a.n_rb % best_R;
+            grid = (long long)best_R * ((a.n_kc + best_cpc - 1) / best_cpc);
             cfg.gridDim = dim3((unsigned)grid);
-            b.fused_reduce = (a.counters != nullptr && debug_env("ELUTQ_DEBUG_FUSED") > 0) ? 1 : 0;
+            b.fused_reduce = (best_cpc == 1 && a.counters != nullptr && debug_env("ELUTQ_DEBUG_FUSED") > 0) ? 1 : 0;
         }
     }
     {   // even rounds: with R = ceil(items/32) rounds, ceil(items/R) warps take items
