@@ -54,6 +54,11 @@ typedef enum elutq_status {
 #define ELUTQ_FLAG_PLAIN_G4    0x10u /* use two 16-entry (g = 4) tables per byte instead of the
                                         fused 256-entry table; same result up to fp32 rounding      */
 
+#define ELUTQ_FLAG_CLUSTER_REDUCE 0x20u /* M = 1, K <= 4096 only: launch one thread-block cluster per row range
+                                           (one CTA per 512-column chunk) and reduce the K split through
+                                           distributed shared memory instead of the workspace + finalize
+                                           kernel; same result bit for bit, measured equally fast          */
+
 #define ELUTQ_HEADER_BYTES 128
 
 /* Human-readable name of a status code (static string, never NULL). */

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     FLAG_OUT_F32,
     FLAG_ACCUMULATE,
     FLAG_PLAIN_G4,
+    FLAG_CLUSTER_REDUCE,
     lib,
     library_path,
     elutq_packed_bytes,

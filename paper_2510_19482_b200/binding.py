@@ -14,6 +14,7 @@ FLAG_OFFSET_ONLY = 0x2
 FLAG_OUT_F32 = 0x4
 FLAG_ACCUMULATE = 0x8
 FLAG_PLAIN_G4 = 0x10
+FLAG_CLUSTER_REDUCE = 0x20
 
 
 class ElutqError(RuntimeError):

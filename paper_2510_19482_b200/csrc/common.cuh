@@ -63,6 +63,8 @@ struct GemmArgs {
                              // CTA b = group * ranges + r, group = `cpc` consecutive chunks
     int cpc;                 // chunks per CTA in the aligned partition
     int fused_reduce;        // 1: the last CTA of a range reduces it in-kernel (needs counters); 0: finalize kernel
+    int cluster_reduce;      // 1: launched as clusters of n_kc CTAs (one per chunk, same row range): partials stay in
+                             //    shared memory and are reduced through distributed shared memory
 };
 
 // Kernel launchers (defined in the .cu files); return a cudaError_t value.
@@ -140,6 +142,19 @@ __device__ __forceinline__ void store_out(const GemmArgs& a, size_t idx, float y
         if (a.flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(Yh[idx]);
         Yh[idx] = __float2half_rn(y);
     }
+}
+// Thread-block cluster helpers (distributed shared memory).
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(const float* local_smem_ptr, unsigned cta_rank) {
+    const uint32_t local = (uint32_t)__cvta_generic_to_shared(local_smem_ptr);
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(cta_rank));
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
 }
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

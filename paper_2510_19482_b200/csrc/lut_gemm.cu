@@ -264,7 +264,7 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
     b.active_warps = kWarps;
-    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1;
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1; b.cluster_reduce = 0;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -300,7 +300,7 @@ int launch_q(const GemmArgs& a, int G, int num_sms, cudaStream_t stream) {
 }  // namespace
 
 int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream) {
-    if (a.flags & ELUTQ_FLAG_PLAIN_G4) return (int)cudaErrorNotSupported;   // decode-kernel variant only
+    if (a.flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE)) return (int)cudaErrorNotSupported;   // decode-kernel variants only
     switch (q) {
         case 1: return launch_q<1>(a, G, num_sms, stream);
         case 2: return launch_q<2>(a, G, num_sms, stream);

@@ -35,6 +35,8 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kTableBytes = 256 * 256;           // 256 entries x 64 columns x 4 bytes
 constexpr int kSmemBytes = kTableBytes + 128;    // + up to 16 group sums + the reduction flag
+constexpr int kClusterPartBytes = 32 * 1024;     // cluster mode: per-CTA partial sums (up to 512 row blocks)
+constexpr int kMaxCluster = 8;
 
 template <int Q, int G>
 struct Cfg {
@@ -127,11 +129,18 @@ __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __rest
 }
 
 // Sum of n partial sums p[0], p[stride], ... in ascending order (the order fixes the rounding, so the
-// result is bit-reproducible); loads are issued 16 at a time so that a reduction costs one or two
+// result is bit-reproducible); loads are issued up to 32 at a time so that a reduction costs one or two
 // L2 round trips instead of one per chunk.
 __device__ __forceinline__ float sum_chunks(const float* p, size_t stride, int n) {
     float sum = 0.f;
     int c = 0;
+    for (; c + 32 <= n; c += 32) {
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __ldcg(p + (size_t)(c + i) * stride);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum += v[i];
+    }
     for (; c + 16 <= n; c += 16) {
         float v[16];
 #pragma unroll
@@ -174,8 +183,9 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     //   flat partition:    one contiguous range of the kc-major item list (jump = 0), cut at chunk ends
     int first, last, jump = 0, range = 0, range_rb0 = 0, range_rb1 = 0;
     if (a.ranges > 0) {
-        const int grp = bid / a.ranges;
-        range = bid - grp * a.ranges;
+        // cluster mode: the n_kc CTAs of a cluster are the chunks of one row range (rank = chunk)
+        const int grp = a.cluster_reduce ? bid % a.n_kc : bid / a.ranges;
+        range = a.cluster_reduce ? bid / a.n_kc : bid - grp * a.ranges;
         range_rb0 = range * a.rb_q + min(range, a.rb_r);
         range_rb1 = range_rb0 + a.rb_q + (range < a.rb_r ? 1 : 0);
         const int kc0 = grp * a.cpc;
@@ -243,6 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
             for (int v = 0; v < C::NSG; ++v)
                 S[u * C::NSG + v] = use_offset ? gsum[C::NSG * (h + 2 * u) + (l / C::W + v) % C::NSG] : 0.f;
 
+        float* cpart = reinterpret_cast<float*>(smem + kTableBytes + 128);   // cluster mode: this CTA's partial sums
         const uint8_t* nvp = nullptr;     // next item's plane vectors / parameter words for this lane
         const uint8_t* npp = nullptr;
         // One item: look-ups, scales, offset term, half-warp combine; with HAS_NEXT the registers of
@@ -296,7 +307,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
             if (a.n_kc == 1) {
                 if (h == 0 && row < a.N) store_out(a, (size_t)row, y);
             } else if (h == 0) {
-                a.partials[(size_t)kc * n_pad + row] = y;
+                if (a.cluster_reduce) cpart[row - range_rb0 * kTileRows] = y;
+                else a.partials[(size_t)kc * n_pad + row] = y;
             }
         };
 
@@ -316,7 +328,25 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         seg = (a.ranges > 0) ? seg + a.n_rb : seg_end;
     }
 
-    if (a.fused_reduce && a.n_kc > 1) {
+    if (a.cluster_reduce && !(a.flags & 0x40000000u)) {
+        // K-split reduction inside the cluster: every CTA holds the partial sums of its chunk for the
+        // cluster's row range in shared memory; after the cluster barrier CTA c adds, for its share of the
+        // rows, the n_kc partials in ascending chunk order (bit-reproducible) straight from its peers'
+        // shared memory.  No workspace, no second kernel.
+        const float* cpart = reinterpret_cast<const float*>(smem + kTableBytes + 128);
+        cluster_barrier();
+        const int rows = (range_rb1 - range_rb0) * kTileRows;
+        const int rank = bid % a.n_kc;
+        const int per = (rows + a.n_kc - 1) / a.n_kc;
+        const int r_end = min(rows, (rank + 1) * per);
+        for (int r = rank * per + tid; r < r_end; r += kThreads) {
+            float sum = 0.f;
+            for (int k = 0; k < a.n_kc; ++k) sum += ld_cluster_f32(cpart + r, (unsigned)k);
+            const int row = range_rb0 * kTileRows + r;
+            if (row < a.N) store_out(a, (size_t)row, sum);
+        }
+        cluster_barrier();          // nobody leaves while a peer may still read its shared memory
+    } else if (a.fused_reduce && a.n_kc > 1) {
         // In-kernel K-split reduction: each CTA publishes its partials and takes one ticket for its row
         // range; the CTA that draws the last ticket of the range adds the chunks in ascending order
         // (bit-reproducible) and writes Y.  The counter wraps to zero, ready for the next call.
@@ -391,7 +421,8 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel<Q, G, PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel<Q, G, PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kSmemBytes + kClusterPartBytes);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
     }
@@ -407,19 +438,53 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
     GemmArgs b = a;
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
     // Aligned partition: groups of `cpc` consecutive chunks x R row ranges, one CTA each.  Pick the cpc
     // that keeps the SMs busiest (work / (SMs * largest CTA share)); fall back to the flat partition
     // of the item list when no choice reaches 80 %.
-    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1;
-    if (a.n_kc > 1 && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1; b.cluster_reduce = 0;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
+    bool use_cluster = false;
+    if (a.n_kc >= 2 && a.n_kc <= kMaxCluster && (a.flags & ELUTQ_FLAG_CLUSTER_REDUCE)) {
+        // Up to 8 chunks: one cluster per row range, one CTA per chunk, reduction through distributed shared memory.
+        int R = (num_sms - 20) / a.n_kc;
+        if (R < 1) R = 1;
+        if (R > a.n_rb) R = a.n_rb;
+        if (debug_env("ELUTQ_DEBUG_R") > 0 && debug_env("ELUTQ_DEBUG_R") < R) R = debug_env("ELUTQ_DEBUG_R");
+        if ((a.n_rb + R - 1) / R * kTileRows * (int)sizeof(float) <= kClusterPartBytes) {
+            cfg.dynamicSmemBytes = kSmemBytes + kClusterPartBytes;
+            cfg.gridDim = dim3((unsigned)(R * a.n_kc));
+            attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+            attr[cfg.numAttrs].val.clusterDim.x = (unsigned)a.n_kc;
+            attr[cfg.numAttrs].val.clusterDim.y = 1;
+            attr[cfg.numAttrs].val.clusterDim.z = 1;
+            cfg.numAttrs += 1;
+            int max_clusters = 0;
+            cudaError_t ce = cudaOccupancyMaxActiveClusters(&max_clusters, lut_gemv_kernel<Q, G, PLAIN>, &cfg);
+            if (ce == cudaSuccess && max_clusters >= 1) {
+                if (R > max_clusters) R = max_clusters;      // one wave of clusters
+                use_cluster = true;
+                b.cluster_reduce = 1;
+                b.ranges = R;
+                b.rb_q = a.n_rb / R;
+                b.rb_r = a.n_rb % R;
+                grid = (long long)R * a.n_kc;
+                cfg.gridDim = dim3((unsigned)grid);
+            } else {
+                (void)cudaGetLastError();
+                cfg.numAttrs -= 1;
+                cfg.dynamicSmemBytes = kSmemBytes;
+                cfg.gridDim = dim3((unsigned)grid);
+            }
+        }
+    }
+    if (!use_cluster && a.n_kc > 1 && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
         // Cost model in item times: the kernel lasts as long as its largest CTA, i.e. that CTA's items
         // plus ~16 item times per table build (measured: an extra build costs far more than the
         // imbalance it could remove).  Minimise that makespan over the aligned choices and the flat one.
@@ -463,11 +528,13 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
         if (b.active_warps > kWarps) b.active_warps = kWarps;
         if (b.active_warps < 1) b.active_warps = 1;
     }
-    if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;   // timing experiment: skip reloads (results invalid)
+    if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;
+    if (debug_env("ELUTQ_DEBUG_SKIP_CLUSTER_REDUCE") > 0) b.flags |= 0x40000000u;   // timing experiment only   // timing experiment: skip reloads (results invalid)
     cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
     count_launch(1);
-    if (e != cudaSuccess || a.n_kc == 1 || b.fused_reduce) return (int)e;
-    return launch_finalize(b, a.n_kc, cfg.numAttrs != 0, stream);
+    if (e != cudaSuccess || a.n_kc == 1 || b.fused_reduce || b.cluster_reduce) return (int)e;
+    if (debug_env("ELUTQ_DEBUG_SKIP_FINALIZE") > 0) return (int)e;   // timing experiment only (Y is not written)
+    return launch_finalize(b, a.n_kc, debug_env("ELUTQ_DEBUG_NO_PDL") == 0, stream);
 }
 
 template <int Q>

@@ -97,6 +97,19 @@ def test_plain_g4_tables_give_the_same_product(q):
     assert hlq.rel_fro_error(y, ref) <= TOL_F32
 
 
+@pytest.mark.parametrize("q,G,N,K", [(2, 128, 1000, 4096), (3, 64, 333, 1536), (4, 128, 5000, 2048)])
+def test_cluster_reduction_variant_is_bit_identical(q, G, N, K):
+    # K <= 4096: the K split can be reduced through distributed shared memory inside one cluster launch
+    layer = workloads.hlq_layer(8, f"cluster/{q}/{N}/{K}", q, G, N, K)
+    X = synth.activations(8, "cluster/x", 1, K)
+    packed = pack_layer(layer)
+    base = gemm_f32(X, packed, N, K)
+    clus = gemm_f32(X, packed, N, K, elutq.FLAG_CLUSTER_REDUCE)
+    assert np.array_equal(base.view(np.uint32), clus.view(np.uint32))
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    assert hlq.rel_fro_error(clus, ref) <= TOL_F32
+
+
 def test_results_are_bit_reproducible_and_workspace_entry_agrees():
     q, G, N, K = 3, 128, 1000, 4096
     layer = workloads.hlq_layer(4, "repro", q, G, N, K)
