@@ -59,6 +59,12 @@ typedef enum elutq_status {
                                            distributed shared memory instead of the workspace + finalize
                                            kernel; same result bit for bit, measured equally fast          */
 
+#define ELUTQ_FLAG_MIRROR 0x40u /* M = 1, G = 128: mirror storage of Appendix D - the weights are read as
+                                   s^_j * b^_j + z^ with b^ = 2b - 1, s^ = s/2, z^ = z + (1/2) sum_j s_j
+                                   (both formed in fp32), the tables hold the +-1 partial sums for the 128
+                                   indices with the top bit clear and the other half is obtained by
+                                   negation; same product up to fp32 rounding                              */
+
 #define ELUTQ_HEADER_BYTES 128
 
 /* Human-readable name of a status code (static string, never NULL). */

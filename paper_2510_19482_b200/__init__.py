@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     FLAG_ACCUMULATE,
     FLAG_PLAIN_G4,
     FLAG_CLUSTER_REDUCE,
+    FLAG_MIRROR,
     lib,
     library_path,
     elutq_packed_bytes,

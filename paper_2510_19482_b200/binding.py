@@ -15,6 +15,7 @@ FLAG_OUT_F32 = 0x4
 FLAG_ACCUMULATE = 0x8
 FLAG_PLAIN_G4 = 0x10
 FLAG_CLUSTER_REDUCE = 0x20
+FLAG_MIRROR = 0x40
 
 
 class ElutqError(RuntimeError):

@@ -126,12 +126,13 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     if (!X || !packed || !Y) return ELUTQ_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
     if ((flags & ELUTQ_FLAG_SKIP_OFFSET) && (flags & ELUTQ_FLAG_OFFSET_ONLY)) return ELUTQ_ERR_INVALID_ARG;
-    if (flags & ~0x3fu) return ELUTQ_ERR_INVALID_ARG;
+    if (flags & ~0x7fu) return ELUTQ_ERR_INVALID_ARG;
+    if ((flags & ELUTQ_FLAG_PLAIN_G4) && (flags & ELUTQ_FLAG_MIRROR)) return ELUTQ_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(packed, 16) || !aligned(Y, 16)) return ELUTQ_ERR_ALIGN;
     BlobMeta m;
     int st = lookup_blob(packed, N, K, &m);
     if (st != ELUTQ_OK) return st;
-    if ((flags & ELUTQ_FLAG_PLAIN_G4) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
+    if ((flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_MIRROR)) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
 
     const size_t cb = counters_bytes(M, N), pb = partials_bytes(M, N, K);
     void* counters = workspace;

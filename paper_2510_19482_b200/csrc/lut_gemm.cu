@@ -300,7 +300,7 @@ int launch_q(const GemmArgs& a, int G, int num_sms, cudaStream_t stream) {
 }  // namespace
 
 int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream) {
-    if (a.flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE)) return (int)cudaErrorNotSupported;   // decode-kernel variants only
+    if (a.flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR)) return (int)cudaErrorNotSupported;   // decode-kernel variants only
     switch (q) {
         case 1: return launch_q<1>(a, G, num_sms, stream);
         case 2: return launch_q<2>(a, G, num_sms, stream);

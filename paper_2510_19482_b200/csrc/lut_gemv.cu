@@ -37,6 +37,9 @@ constexpr int kTableBytes = 256 * 256;           // 256 entries x 64 columns x 4
 constexpr int kSmemBytes = kTableBytes + 128;    // + up to 16 group sums + the reduction flag
 constexpr int kClusterPartBytes = 32 * 1024;     // cluster mode: per-CTA partial sums (up to 512 row blocks)
 constexpr int kMaxCluster = 8;
+constexpr int kModeFused = 0;      // 256-entry 0/1 tables (default)
+constexpr int kModePlainG4 = 1;    // two 16-entry g = 4 tables per byte
+constexpr int kModeMirror = 2;     // Appendix D mirror storage: 128-entry +-1 tables, sign applied on look-up
 
 template <int Q, int G>
 struct Cfg {
@@ -68,7 +71,7 @@ __device__ __forceinline__ void load_item(Item<Q, G>& it, const uint8_t* vp, con
 // lane -> column pair (2*lane, 2*lane+1); warp -> high nibble hi = warp & 15 and low-nibble half
 // lh = warp >> 4 (entries lo = 8*lh .. 8*lh+7).  Both columns are computed with packed fp32x2
 // adds and stored with one 64-bit store per entry pair (conflict-free: 256 contiguous bytes per warp).
-template <int G, bool PLAIN>
+template <int G, int MODE>
 __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __restrict__ X, int kc, int K, int tid) {
     constexpr int W = G / 8;
     float* gsum = reinterpret_cast<float*>(smem + kTableBytes);
@@ -107,21 +110,29 @@ __device__ __forceinline__ void build_tables(uint8_t* smem, const __half* __rest
         if ((hi >> b) & 1) Bv = fadd2(Bv, x[4 + b]);
     float2* row = reinterpret_cast<float2*>(smem) + (size_t)(hi * 16 + lh * 8) * 32 + lane;
     float2 e7 = make_float2(0.f, 0.f);
+    // mirror mode (Appendix D): entries are sums of +-x_i (+ where the index bit is set), i.e.
+    // 2 * (0/1 sum) - (sum of all 8 activations); only indices with bit 7 clear (hi < 8) are stored
+    float2 negsx = make_float2(0.f, 0.f);
+    if (MODE == kModeMirror) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) negsx = fadd2(negsx, make_float2(-x[i].x, -x[i].y));
+    }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         float2 e;
-        if (PLAIN) {
+        if (MODE == kModePlainG4) {
             // unfused variant: entry p holds A[lo] in rows with hi == 0 and B[hi] in rows with lo == 0
             const float2 zero = make_float2(0.f, 0.f);
             e = (hi == 0) ? A[t] : ((lh == 0 && t == 0) ? Bv : zero);
         } else {
             e = fadd2(A[t], Bv);
+            if (MODE == kModeMirror) e = fadd2(fadd2(e, e), negsx);
         }
-        row[t * 32] = e;
+        if (MODE != kModeMirror || hi < 8) row[t * 32] = e;
         if (t == 7) e7 = fadd2(A[t], Bv);
     }
     if (warp == 31) {                                  // hi = 15, lo = 15: entry 255 = sum of the column's 8 activations
-        float total = e7.x + e7.y;
+        float total = (MODE == kModeMirror) ? -(negsx.x + negsx.y) : e7.x + e7.y;
 #pragma unroll
         for (int off = W / 4; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
         if ((lane % (W / 2)) == 0) gsum[lane / (W / 2)] = total;
@@ -168,7 +179,7 @@ __device__ __forceinline__ float sum_chunks(const float* p, size_t stride, int n
     return sum;
 }
 
-template <int Q, int G, bool PLAIN>
+template <int Q, int G, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a) {
     using C = Cfg<Q, G>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -243,7 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         const int kc = seg / a.n_rb;
         const int seg_end = (a.ranges > 0) ? seg + seg_len0 : min(last, (kc + 1) * a.n_rb);
         __syncthreads();
-        build_tables<G, PLAIN>(smem, a.X, kc, a.K, tid);
+        build_tables<G, MODE>(smem, a.X, kc, a.K, tid);
         __syncthreads();
 
         float S[C::GL];
@@ -251,7 +262,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         for (int u = 0; u < 2; ++u)
 #pragma unroll
             for (int v = 0; v < C::NSG; ++v)
-                S[u * C::NSG + v] = use_offset ? gsum[C::NSG * (h + 2 * u) + (l / C::W + v) % C::NSG] : 0.f;
+                S[u * C::NSG + v] = (use_offset || MODE == kModeMirror) ? gsum[C::NSG * (h + 2 * u) + (l / C::W + v) % C::NSG] : 0.f;
 
         float* cpart = reinterpret_cast<float*>(smem + kTableBytes + 128);   // cluster mode: this CTA's partial sums
         const uint8_t* nvp = nullptr;     // next item's plane vectors / parameter words for this lane
@@ -268,6 +279,21 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
                 prm[2 * i + 1] = f.y;
             }
             if (HAS_NEXT) static_for<0, C::NPW>([&](auto i) { buf.p[i] = ldg_stream_u32<i * 128>(npp); });
+            if (MODE == kModeMirror) {
+                // s^ = s / 2 and z^ = z + (1/2) sum_j s_j, formed in fp32 (exact halving, one rounding for z^)
+#pragma unroll
+                for (int gi = 0; gi < C::GL; ++gi) {
+                    float half_sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < Q; ++j) {
+                        prm[gi * (Q + 1) + j] *= 0.5f;
+                        half_sum += prm[gi * (Q + 1) + j];
+                    }
+                    // the group-sum term carries z (unless the offset is skipped) and, when the planes are
+                    // used, the (1/2) sum_j s_j that the +-1 rewrite moves out of the look-ups
+                    prm[gi * (Q + 1) + Q] = (use_offset ? prm[gi * (Q + 1) + Q] : 0.f) + (use_planes ? half_sum : 0.f);
+                }
+            }
             float y = 0.f;
             if (use_planes) {
                 static_for<0, 2 * Q>([&](auto uj) {
@@ -284,8 +310,13 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
                                 const int i = v * C::W + ii + t;
                                 // address = (weight byte << 8) | lane column
                                 const uint32_t off = prmt(wd[i >> 2], colp[i >> 2], 0xCC04 + 0x11 * (i & 3));
-                                if (!PLAIN) {
+                                if (MODE == kModeFused) {
                                     e[t] = *reinterpret_cast<const float*>(smem + off + u * 128);
+                                } else if (MODE == kModeMirror) {
+                                    // index bit 7 set: read the complemented index and negate (the +-1 table is antisymmetric)
+                                    const uint32_t m = prmt(wd[i >> 2], colp[i >> 2], 0xCC8C + 0x10 * (i & 3));   // 0xFF00 or 0
+                                    const float tv = *reinterpret_cast<const float*>(smem + (off ^ m) + u * 128);
+                                    e[t] = __uint_as_float(__float_as_uint(tv) ^ ((m << 16) & 0x80000000u));
                                 } else {
                                     e[t] = *reinterpret_cast<const float*>(smem + (off & 0x0fffu) + u * 128)     // low nibble table
                                          + *reinterpret_cast<const float*>(smem + (off & 0xf0ffu) + u * 128);    // high nibble table
@@ -415,13 +446,13 @@ int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stre
 
 namespace {
 
-template <int Q, int G, bool PLAIN>
+template <int Q, int G, int MODE>
 int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel<Q, G, PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel<Q, G, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmemBytes + kClusterPartBytes);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
@@ -466,7 +497,7 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
             attr[cfg.numAttrs].val.clusterDim.z = 1;
             cfg.numAttrs += 1;
             int max_clusters = 0;
-            cudaError_t ce = cudaOccupancyMaxActiveClusters(&max_clusters, lut_gemv_kernel<Q, G, PLAIN>, &cfg);
+            cudaError_t ce = cudaOccupancyMaxActiveClusters(&max_clusters, lut_gemv_kernel<Q, G, MODE>, &cfg);
             if (ce == cudaSuccess && max_clusters >= 1) {
                 if (R > max_clusters) R = max_clusters;      // one wave of clusters
                 use_cluster = true;
@@ -530,7 +561,7 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     }
     if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;
     if (debug_env("ELUTQ_DEBUG_SKIP_CLUSTER_REDUCE") > 0) b.flags |= 0x40000000u;   // timing experiment only   // timing experiment: skip reloads (results invalid)
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, PLAIN>, b);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, MODE>, b);
     count_launch(1);
     if (e != cudaSuccess || a.n_kc == 1 || b.fused_reduce || b.cluster_reduce) return (int)e;
     if (debug_env("ELUTQ_DEBUG_SKIP_FINALIZE") > 0) return (int)e;   // timing experiment only (Y is not written)
@@ -540,11 +571,12 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
 template <int Q>
 int launch_q(const GemmArgs& a, int G, int num_sms, cudaStream_t stream) {
     switch (G) {
-        case 32: return launch_one<Q, 32, false>(a, num_sms, stream);
-        case 64: return launch_one<Q, 64, false>(a, num_sms, stream);
+        case 32: return launch_one<Q, 32, kModeFused>(a, num_sms, stream);
+        case 64: return launch_one<Q, 64, kModeFused>(a, num_sms, stream);
         case 128:
-            return (a.flags & ELUTQ_FLAG_PLAIN_G4) ? launch_one<Q, 128, true>(a, num_sms, stream)
-                                                   : launch_one<Q, 128, false>(a, num_sms, stream);
+            if (a.flags & ELUTQ_FLAG_PLAIN_G4) return launch_one<Q, 128, kModePlainG4>(a, num_sms, stream);
+            if (a.flags & ELUTQ_FLAG_MIRROR) return launch_one<Q, 128, kModeMirror>(a, num_sms, stream);
+            return launch_one<Q, 128, kModeFused>(a, num_sms, stream);
         default: return (int)cudaErrorInvalidValue;
     }
 }

@@ -97,6 +97,25 @@ def test_plain_g4_tables_give_the_same_product(q):
     assert hlq.rel_fro_error(y, ref) <= TOL_F32
 
 
+@pytest.mark.parametrize("q,N,K", [(2, 333, 1536), (3, 1000, 4096), (4, 64, 2560), (1, 50, 512)])
+def test_mirror_storage_variant_matches_oracle(q, N, K):
+    # Appendix D: +-1 bits, s^ = s/2, z^ = z + sum(s)/2, half-size antisymmetric tables
+    from oracle import lut
+    G = 128
+    layer = workloads.hlq_layer(9, f"mirror/{q}/{N}/{K}", q, G, N, K, signed_scales=True)
+    X = synth.activations(9, "mirror/x", 1, K, outliers=True)
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    ref_mirror = lut.mirror_lut_matmul(X, layer.planes, layer.scales, layer.offsets, G, g=8)
+    y = gemm_f32(X, packed, N, K, elutq.FLAG_MIRROR)
+    assert hlq.rel_fro_error(y, ref) <= 2 * TOL_F32
+    assert hlq.rel_fro_error(y, ref_mirror) <= 2 * TOL_F32
+    ys = gemm_f32(X, packed, N, K, elutq.FLAG_MIRROR | elutq.FLAG_SKIP_OFFSET)
+    # without the offset term the mirror form still carries (1/2) sum_j s_j * sum(x) of the +-1 rewrite:
+    # it must equal the plain scale term
+    assert hlq.rel_fro_error(ys, hlq.scale_term(X, layer.planes, layer.scales, G)) <= 1e-4
+
+
 @pytest.mark.parametrize("q,G,N,K", [(2, 128, 1000, 4096), (3, 64, 333, 1536), (4, 128, 5000, 2048)])
 def test_cluster_reduction_variant_is_bit_identical(q, G, N, K):
     # K <= 4096: the K split can be reduced through distributed shared memory inside one cluster launch
