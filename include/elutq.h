@@ -65,6 +65,12 @@ typedef enum elutq_status {
                                    indices with the top bit clear and the other half is obtained by
                                    negation; same product up to fp32 rounding                              */
 
+#define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 64: stay on the look-up-table kernels.  Without this flag batches of
+                                     64 rows or more (G = 128) take the dequantise-and-contract path: the
+                                     weight tile is rebuilt in fp16 from the bit-planes (BCQ form of
+                                     Appendix D) and contracted on the tensor cores with fp32 accumulation;
+                                     its results carry the fp16 rounding of W_hat (about 3e-4 relative)     */
+
 #define ELUTQ_HEADER_BYTES 128
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -191,6 +197,13 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
  *     GPU, e.g. on different streams, race on it: keep them stream-ordered.
  */
 int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
+
+/*
+ * Device-side status of the library-owned scratch of `stream` (synchronises the stream).
+ * *status is 0 unless a kernel gave up on a bounded wait (then a non-zero code that stays set
+ * until elutq_release_scratch).  Kernels never spin without a limit.
+ */
+int elutq_device_status(void* stream, int* status);
 
 /* Number of kernel launches the library has issued in this process (all entry
  * points); lets a benchmark count its launches. */

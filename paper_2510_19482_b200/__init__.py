@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     FLAG_PLAIN_G4,
     FLAG_CLUSTER_REDUCE,
     FLAG_MIRROR,
+    FLAG_LUT_ONLY,
     lib,
     library_path,
     elutq_packed_bytes,
@@ -29,6 +30,7 @@ from .binding import (  # noqa: F401
     elutq_lut_gemm_ws,
     elutq_lut_gemm_host,
     elutq_lut_gemm_static,
+    elutq_device_status,
     elutq_launch_count,
     elutq_release_scratch,
     elutq_status_string,

@@ -16,6 +16,7 @@ FLAG_ACCUMULATE = 0x8
 FLAG_PLAIN_G4 = 0x10
 FLAG_CLUSTER_REDUCE = 0x20
 FLAG_MIRROR = 0x40
+FLAG_LUT_ONLY = 0x80
 
 
 class ElutqError(RuntimeError):
@@ -46,6 +47,7 @@ _SIGNATURES = {
     "elutq_lut_gemm_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p, c_size_t, c_void_p]),
     "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_lut_gemm_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
 }
@@ -171,3 +173,10 @@ def elutq_lut_gemm_static(X, packed, Y, M: int, N: int, K: int, stream=None) -> 
     """elutq_lut_gemm for callers that must not allocate: scratch is a fixed 4 MiB array inside the library."""
     _check(lib().elutq_lut_gemm_static(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, _stream(stream)),
            "elutq_lut_gemm_static")
+
+
+def elutq_device_status(stream=None) -> int:
+    """0 unless a kernel gave up on a bounded wait (synchronises the stream)."""
+    out = c_int(0)
+    _check(lib().elutq_device_status(_stream(stream), ctypes.byref(out)), "elutq_device_status")
+    return out.value

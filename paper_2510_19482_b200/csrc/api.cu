@@ -126,7 +126,7 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     if (!X || !packed || !Y) return ELUTQ_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
     if ((flags & ELUTQ_FLAG_SKIP_OFFSET) && (flags & ELUTQ_FLAG_OFFSET_ONLY)) return ELUTQ_ERR_INVALID_ARG;
-    if (flags & ~0x7fu) return ELUTQ_ERR_INVALID_ARG;
+    if (flags & ~0xffu) return ELUTQ_ERR_INVALID_ARG;
     if ((flags & ELUTQ_FLAG_PLAIN_G4) && (flags & ELUTQ_FLAG_MIRROR)) return ELUTQ_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(packed, 16) || !aligned(Y, 16)) return ELUTQ_ERR_ALIGN;
     BlobMeta m;
@@ -161,7 +161,9 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     a.flags = flags;
     const int sms = num_sms();
     int ce;
+    const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY;
     if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
+    else if (M >= 64 && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
     else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);
     if (ce != 0) return cuda_fail((cudaError_t)ce);
     return ELUTQ_OK;
@@ -308,6 +310,28 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host, in
     if (st != ELUTQ_OK) return st;
     e = cudaMemcpyAsync(Y_host, yd, yb, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e);
+    return ELUTQ_OK;
+}
+
+int elutq_device_status(void* stream, int* status) {
+    if (!status) return ELUTQ_ERR_INVALID_ARG;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    void* ptr = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_scratch.find(std::make_tuple(dev, stream, 0));
+        if (it != g_scratch.end()) ptr = it->second.ptr;
+    }
+    *status = 0;
+    e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ptr) return ELUTQ_OK;
+    unsigned word = 0;
+    e = cudaMemcpy(&word, ptr, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *status = (int)word;
     return ELUTQ_OK;
 }
 

@@ -74,6 +74,7 @@ int launch_unpack(const uint8_t* packed, const Geo& g, uint8_t* planes, __half* 
                   __half* offsets, cudaStream_t stream);
 int launch_lut_gemv(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
+int launch_hlq_mma(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 
 int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream);
 int debug_env(const char* name);

@@ -1,0 +1,75 @@
+"""GPU parity of the tensor-core (dequantise-and-contract) path for batches of 64 rows or more.
+
+Tolerance: the path rebuilds W_hat in fp16 (the BCQ form: z^ rounded once, then one fused multiply-add
+per plane, each rounding at 2^-11 relative), multiplies exactly and accumulates in fp32.  The weight
+rounding errors are independent across k, so the relative Frobenius error of Y is about 2^-12..2^-11
+(2.5e-4 .. 5e-4) before the output rounding; the bar is the benchmark's 1e-3.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_19482_b200 as elutq
+import workloads
+from oracle import hlq
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import gemm_f16, gemm_f32, pack_layer, x_dev  # noqa: E402
+
+TOL = 1e-3
+
+# (q, N, K, M): one tile, ragged N / M / K tails, every q, several token tiles, a K split
+CASES = [(2, 256, 512, 64), (2, 200, 1024, 100), (3, 1000, 1536, 128), (4, 384, 2560, 300),
+         (1, 130, 640, 65), (2, 4096, 4096, 128), (3, 512, 4096, 700)]
+
+
+@pytest.mark.parametrize("q,N,K,M", CASES)
+def test_tensor_core_path_matches_oracle(q, N, K, M):
+    G = 128
+    layer = workloads.hlq_layer(30, f"mma/{q}/{N}/{K}", q, G, N, K, signed_scales=(q == 3))
+    X = synth.activations(30, f"mma/x/{M}/{K}", M, K, outliers=(q == 2))
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    y32 = gemm_f32(X, packed, N, K)
+    assert elutq.elutq_device_status() == 0
+    assert np.all(np.isfinite(y32))
+    assert hlq.rel_fro_error(y32, ref) <= TOL
+    worst_row = max(hlq.rel_fro_error(y32[m], ref[m]) for m in range(0, M, max(1, M // 16)))
+    assert worst_row <= 2 * TOL
+    y16 = gemm_f16(X, packed, N, K)
+    assert hlq.rel_fro_error(y16, ref) <= TOL
+    # the look-up-table kernels on the same batch agree with it within the same bar
+    ylut = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)
+    assert hlq.rel_fro_error(ylut, ref) <= 5e-6
+    assert hlq.rel_fro_error(y32, ylut) <= TOL
+
+
+def test_tensor_core_path_terms_and_accumulate():
+    q, G, N, K, M = 2, 128, 300, 1024, 96
+    layer = workloads.hlq_layer(31, "mma/flags", q, G, N, K)
+    X = synth.activations(31, "mma/flags/x", M, K)
+    packed = pack_layer(layer)
+    ys = gemm_f32(X, packed, N, K, elutq.FLAG_SKIP_OFFSET)
+    yb = gemm_f32(X, packed, N, K, elutq.FLAG_OFFSET_ONLY)
+    yf = gemm_f32(X, packed, N, K)
+    assert hlq.rel_fro_error(ys, hlq.scale_term(X, layer.planes, layer.scales, G)) <= TOL
+    assert hlq.rel_fro_error(yb, hlq.offset_term(X, layer.offsets, G)) <= TOL
+    assert hlq.rel_fro_error(yf, hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)) <= TOL
+    Y = torch.full((M, N), 1.5, dtype=torch.float32, device="cuda")
+    elutq.elutq_lut_gemm_f32(x_dev(X), packed, Y, M, N, K, elutq.FLAG_ACCUMULATE)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(Y.cpu().numpy(), yf + 1.5, rtol=0, atol=1e-5 * np.abs(yf).max())
+    assert elutq.elutq_device_status() == 0
+
+
+def test_tensor_core_path_is_bit_reproducible():
+    q, G, N, K, M = 3, 128, 512, 2048, 128
+    layer = workloads.hlq_layer(32, "mma/repro", q, G, N, K)
+    X = synth.activations(32, "mma/repro/x", M, K)
+    packed = pack_layer(layer)
+    a = gemm_f16(X, packed, N, K)
+    b = gemm_f16(X, packed, N, K)
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
