@@ -4,20 +4,29 @@
 // weight byte), while Y = X W_hat^T is then a genuine dense contraction.  This kernel rebuilds each
 // weight tile in fp16 from the packed bit-planes and runs it through tcgen05.mma:
 //
-//   CTA tile   128 weight rows (UMMA M) x NT tokens (UMMA N = 64, 128 or 256), K walked in steps of 256
-//              (half a packed tile: super-groups 2u and 2u+1 of a 512-column chunk)
-//   A operand  W_hat tile, 128 x 256 fp16, K-major, no swizzle: core matrices of 8 rows x 16 bytes,
-//              [row group][k8] order (leading byte offset 128, stride byte offset 4096).  One warp
-//              dequantises one packed item (16 rows): lane (h, l) owns row l and super-group h, and every
-//              packed byte (8 consecutive k of one row) becomes exactly one 16-byte core-matrix row.
-//   dequant    the BCQ / mirror form of Appendix D: W_hat = z^ + sum_j (-s_j/2) * (+-1), where the +-1.0
-//              fp16 operand is built by dropping the weight bit into the sign position of 1.0 - two
-//              integer instructions and one HFMA2 per pair of weights and plane.  z^ = z + (1/2) sum s_j
-//              is formed in fp32 and rounded once.
-//   B operand  X tile, NT x 256 fp16, same canonical layout
-//   D          fp32 in tensor memory (128 lanes x NT columns); read back with tcgen05.ld, then either
-//              written to Y (one rounding to fp16) or, with a K split, to the fp32 partial buffer that the
-//              shared finalize kernel reduces in ascending order.
+//   CTA tile   TT x 128 tokens (UMMA M = 128, TT = 1 or 2 accumulators) x NW weight rows (UMMA N = 128
+//              or 256), K walked in steps of 128 (one super-group of a 512-column chunk).  Weight rows are
+//              the wide dimension on purpose: a packed weight is 8x smaller than an fp16 activation, so the
+//              activation tile is what the L2 has to feed again and again; two token tiles share one
+//              dequantised weight tile, which halves both the dequantisation work and the weight traffic.
+//   A operand  X tile, 128 tokens x 128 k fp16, K-major with the 128-byte swizzle: two blocks of 64 k, a
+//              token row is 128 contiguous bytes whose 16-byte chunks are XOR-ed with (token mod 8).  A
+//              quarter-warp copies the 8 chunks of one token: four full 32-byte sectors on the global side,
+//              eight different bank groups on the shared side.  Two stages, filled by cp.async one step
+//              ahead of the MMAs that read them.
+//   B operand  W_hat tile, NW x 128 fp16, K-major without swizzle: core matrices of 8 rows x 16 bytes in
+//              [row group][k8] order (leading byte offset 128, stride byte offset 2048).  A warp
+//              dequantises two packed items (32 rows): lane 16*i + l owns row l of item i and the step's
+//              super-group, and every packed byte (8 consecutive k of one row) becomes exactly one 16-byte
+//              core-matrix row.
+//   dequant    the BCQ / mirror form of Appendix D: W_hat = z^ + sum_j (-s_j/2) * (+-1).  The +-1.0 fp16
+//              factors of a plane byte (8 weights) come from a 256-entry shared-memory table, one 16-byte
+//              load per byte and plane, followed by four HFMA2.  z^ = z + (1/2) sum s_j is formed in fp32
+//              and rounded once.
+//   D          fp32 in tensor memory (lane = token, column = weight row, one block of NW columns per token
+//              tile); read back with tcgen05.ld, then either written to Y (one rounding to fp16, 16-byte
+//              stores) or, with a K split, to the fp32 partial buffer that the shared finalize kernel
+//              reduces in ascending order.
 //
 // Every wait is bounded: if the MMA-completion barrier does not flip within the limit the CTA raises the
 // status word, skips the remaining work, still releases its tensor memory and returns.
@@ -28,18 +37,25 @@ namespace elutq {
 namespace {
 
 constexpr int kMmaThreads = 256;
-constexpr int kTileN = 128;                 // weight rows per CTA (UMMA M)
-constexpr int kStepK = 256;                 // K per step
-constexpr int kABytes = kTileN * kStepK * 2;
+constexpr int kTileM = 128;                  // tokens per accumulator (UMMA M)
+constexpr int kStepK = 128;                  // K per step
+constexpr int kXTileBytes = kTileM * kStepK * 2;   // one token tile of one step: 2 blocks of [128 tokens][128 bytes]
+constexpr int kXStages = 2;
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr int kSignTableBytes = 256 * 128;   // 256 byte values x 8 bank-group replicas x 16 bytes
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// K-major, no-swizzle shared-memory matrix descriptor: start address, leading (K) and stride (row group)
-// byte offsets in 16-byte units, descriptor version 1.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
-    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(128u >> 4) << 16) | ((uint64_t)(4096u >> 4) << 32) |
+// Shared-memory matrix descriptors (version 1).  Addresses and offsets are in 16-byte units.
+// K-major, no swizzle: leading (K direction) offset 128 bytes, stride (row group) offset 2048 bytes.
+__device__ __forceinline__ uint64_t desc_noswizzle(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(128u >> 4) << 16) | ((uint64_t)(2048u >> 4) << 32) |
            ((uint64_t)1 << 46);
+}
+// K-major, 128-byte swizzle: rows of 128 bytes, row groups of 1024 bytes; the leading offset is not used.
+__device__ __forceinline__ uint64_t desc_swizzle128(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024u >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -54,36 +70,86 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 
-template <int Q, int NT>
-__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits) {
-    constexpr int NPW = 2 * (Q + 1) / 2 + ((2 * (Q + 1)) % 2);      // parameter words per lane at G = 128: Q + 1
+// 32 consecutive outputs of one token row: Y (fp16 or fp32, optionally accumulating) or the fp32 partials.
+__device__ __forceinline__ void store_row32(const GemmArgs& a, int m, int n0, const uint32_t (&r)[32], int splits,
+                                            int split, size_t n_pad, bool y_vec_ok) {
+    if (splits > 1) {
+        float* dst = a.partials + ((size_t)split * a.M + m) * n_pad + n0;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+            if ((size_t)(n0 + i) < n_pad)
+                *reinterpret_cast<uint4*>(dst + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+        return;
+    }
+    if (y_vec_ok) {                        // fp16 output, no accumulation, N a multiple of 8, Y 16-byte aligned
+        __half* dst = reinterpret_cast<__half*>(a.Y) + (size_t)m * a.N + n0;
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+            if (n0 + i < a.N) {
+                uint32_t p[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const __half2 v = __floats2half2_rn(__uint_as_float(r[i + 2 * t]), __uint_as_float(r[i + 2 * t + 1]));
+                    p[t] = *reinterpret_cast<const uint32_t*>(&v);
+                }
+                *reinterpret_cast<uint4*>(dst + i) = make_uint4(p[0], p[1], p[2], p[3]);
+            }
+        }
+        return;
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (n0 + i < a.N) store_out(a, (size_t)m * a.N + n0 + i, __uint_as_float(r[i]));
+}
+
+// NW = weight rows per CTA (UMMA N: 128 or 256); TT = token tiles of 128 per CTA (1 or 2).
+template <int Q, int NW, int TT>
+__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits, const int dbg) {
+    constexpr int NPW = Q + 1;                           // parameter words per lane at G = 128
     constexpr int PLANE_BYTES = 1024 * Q;
     constexpr int TILE_BYTES = PLANE_BYTES + 128 * (Q + 1);
+    constexpr int PAIRS = NW / 32;                       // item pairs per step: 8 or 4
+    constexpr int WPP = (kMmaThreads / 32) / PAIRS;      // warps sharing one item pair: 1 or 2
+    constexpr int NB = 16 / WPP;                         // plane bytes per lane and step
+    constexpr int X_STAGE_BYTES = TT * kXTileBytes;
+    constexpr int W_BYTES = NW * kStepK * 2;
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint8_t* sA = smem;
-    uint8_t* sB = smem + kABytes;
-    uint64_t* mbar = reinterpret_cast<uint64_t*>(smem + kABytes + NT * kStepK * 2);
+    uint8_t* sX = smem;                                  // A operand stages
+    uint8_t* sW = smem + kXStages * X_STAGE_BYTES;       // B operand
+    uint8_t* sT = sW + W_BYTES;                          // sign table
+    uint64_t* mbar = reinterpret_cast<uint64_t*>(sT + kSignTableBytes);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 1);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int h = lane >> 4, l = lane & 15;
+    const int l = lane & 15;
     const int n_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
-    const int m0 = m_tile * NT;
-    const int n_steps = 2 * a.n_kc;                                   // half chunks
+    const int m0 = m_tile * (TT * kTileM);
+    const int n_steps = 4 * a.n_kc;                                   // super-groups
     const int step0 = (int)((long long)n_steps * split / splits);
     const int step1 = (int)((long long)n_steps * (split + 1) / splits);
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
-    // ---- set-up: tensor memory, completion barrier --------------------------------------------
+    // ---- set-up: tensor memory, completion barrier, sign table ---------------------------------
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)NT) : "memory");
+                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)(TT * NW)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // Sign table: entry b holds, for the 8 bits of a plane byte, fp16 +1.0 (bit clear) or -1.0 (bit set),
+    // i.e. the eight +-1 factors of one core-matrix row.  Each entry is stored 8 times, once per 16-byte
+    // bank group, and a lane reads replica (lane & 7): the 8 lanes of a quarter-warp never collide.
+    for (int e = tid; e < 256 * 8; e += kMmaThreads) {
+        const int b = e >> 3;
+        uint32_t w4[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            w4[i] = (((b >> (2 * i)) & 1) ? 0xBC00u : 0x3C00u) | ((((b >> (2 * i + 1)) & 1) ? 0xBC00u : 0x3C00u) << 16);
+        *reinterpret_cast<uint4*>(sT + e * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -93,182 +159,222 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     grid_launch_dependents();
     grid_dependency_wait();
 
-    // instruction descriptor: D = fp32, A = B = fp16, both K-major, N = NT, M = 128
-    constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
-    const uint32_t a_addr = smem_u32(sA), b_addr = smem_u32(sB), bar_addr = smem_u32(mbar);
+    // instruction descriptor: D = fp32, A = B = fp16, both K-major, M = 128 tokens, N = NW weight rows
+    constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NW >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    const uint32_t x_addr = smem_u32(sX), w_addr = smem_u32(sW), bar_addr = smem_u32(mbar);
 
-    const int rb = n_tile * (kTileN / kTileRows) + warp;               // this warp's row block
-    const bool rb_valid = rb < a.n_rb;
-    // destination of this lane's core-matrix rows: row group 2*warp + l/8, row l%8; column added per byte
-    const uint32_t a_row_off = (uint32_t)((2 * warp + (l >> 3)) * 32) * 128u + (uint32_t)(l & 7) * 16u;
+    // Asynchronous copy of the activation tile(s) of one step into a stage.  Thread (token r = tid / 8 + 32 p,
+    // chunk j = tid % 8): 16 bytes at k = step*128 + kb*64 + 8 j, stored at chunk j ^ (r & 7) of row r.
+    auto copy_x = [&](int step, int stage) {
+        if (dbg & 1) return;
+        const int j = tid & 7, r0 = tid >> 3;
+        const uint32_t dst0 = x_addr + (uint32_t)stage * X_STAGE_BYTES + (uint32_t)r0 * 128u + (uint32_t)((j ^ (r0 & 7)) * 16);
+#pragma unroll
+        for (int tt = 0; tt < TT; ++tt) {
+#pragma unroll
+            for (int kb = 0; kb < 2; ++kb) {
+                const int k = step * kStepK + kb * 64 + j * 8;
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const int m = m0 + tt * kTileM + p * 32 + r0;                 // (r0 + 32 p) & 7 == r0 & 7
+                    const uint32_t dst = dst0 + (uint32_t)(tt * kXTileBytes + kb * (kTileM * 128) + p * 32 * 128);
+                    if (k < a.K && m < a.M) {
+                        const __half* src = a.X + (size_t)m * a.K + k;
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(src) : "memory");
+                    } else {
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" :: "r"(dst), "r"(0u) : "memory");
+                    }
+                }
+            }
+        }
+    };
+
+    // Weights of the current step live in registers; the next step's are requested while this one is dequantised.
+    // Lane 16 i + l reads what packed lane (h, l) of item i owns: plane vectors of half u, parameter words.
+    const int pair = warp % PAIRS;                        // item pair of this warp
+    const int bsel = warp / PAIRS;                        // which NB bytes of the 16 (only when two warps share a pair)
+    const int item = 2 * pair + (lane >> 4);
+    const int rb = n_tile * (NW / kTileRows) + item;
+    uint4 vec[Q];
+    uint32_t pw[NPW];
+    auto load_weights = [&](int step) {
+        const int kc = step >> 2, sg = step & 3, h = sg & 1, u = sg >> 1;
+        if (rb < a.n_rb) {
+            const uint8_t* tile = a.tiles + ((size_t)kc * a.n_rb + rb) * TILE_BYTES;
+            const int pl = 16 * h + l;
+            static_for<0, Q>([&](auto j) { vec[j] = ldg_stream_v4<0>(tile + ((u * Q + j) * 32 + pl) * 16); });
+            static_for<0, NPW>([&](auto i) { pw[i] = ldg_stream_u32<0>(tile + PLANE_BYTES + (i * 32 + pl) * 4); });
+        }
+    };
 
     uint32_t phase = 0;
     bool ok = true;
-    for (int step = step0; step < step1 && ok; ++step) {
-        const int kc = step >> 1, u = step & 1;
+    if (step0 < step1) {
+        copy_x(step0, 0);
+        load_weights(step0);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
 
-        // ---- A: dequantise this warp's item half into the core-matrix layout ----------------------
-        if (rb_valid && use_planes | use_offset) {
-            const uint8_t* tile = a.tiles + ((size_t)kc * a.n_rb + rb) * TILE_BYTES;
-            uint4 vec[Q];
-            uint32_t pw[NPW];
-            static_for<0, Q>([&](auto j) { vec[j] = ldg_stream_v4<0>(tile + ((u * Q + j) * 32 + lane) * 16); });
-            static_for<0, NPW>([&](auto i) { pw[i] = ldg_stream_u32<0>(tile + PLANE_BYTES + (i * 32 + lane) * 4); });
-            // record of this half: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
-            float sc[Q + 1];
+    for (int step = step0; step < step1 && ok; ++step) {
+        const int stage = (step - step0) & 1;
+        if (step > step0 && !(dbg & 4)) {
+            // the tensor core must be done with the weight tile and with the other activation stage
+            ok = __syncthreads_and(mbar_wait(bar_addr, phase) ? 1 : 0) != 0;   // one decision for the whole CTA
+            phase ^= 1u;
+            if (!ok) break;
+        }
+        if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+
+        // ---- B operand: dequantise this lane's row of the step's super-group into the core-matrix layout ----
+        if (!(dbg & 2)) {
+            const int u = (step & 3) >> 1;
+            const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 16) * 128u + (uint32_t)(l & 7) * 16u;
+            if (rb < a.n_rb && (use_planes | use_offset)) {
+                // parameter record of this super-group: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
+                float sc[Q + 1];
 #pragma unroll
-            for (int c = 0; c <= Q; ++c) {
-                float lo_v = 0.f, hi_v = 0.f;
+                for (int c = 0; c <= Q; ++c) {
+                    float lo_v = 0.f, hi_v = 0.f;
 #pragma unroll
-                for (int uu = 0; uu < 2; ++uu) {
-                    const int e = uu * (Q + 1) + c;
-                    const uint32_t wv = pw[e >> 1];
-                    const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
-                    if (uu == 0) lo_v = f; else hi_v = f;
+                    for (int uu = 0; uu < 2; ++uu) {
+                        const int e = uu * (Q + 1) + c;
+                        const uint32_t wv = pw[e >> 1];
+                        const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
+                        if (uu == 0) lo_v = f; else hi_v = f;
+                    }
+                    sc[c] = u ? hi_v : lo_v;
                 }
-                sc[c] = u ? hi_v : lo_v;
-            }
-            float zhat = use_offset ? sc[Q] : 0.f;
-            __half2 sneg[Q];
-#pragma unroll
-            for (int j = 0; j < Q; ++j) {
-                const float sj = use_planes ? sc[j] : 0.f;
-                zhat += 0.5f * sj;
-                sneg[j] = __float2half2_rn(-0.5f * sj);               // exact halving of an fp16 value
-            }
-            const __half2 z2 = __float2half2_rn(zhat);
-            const uint32_t kSign = 0x80008000u, kOne = 0x3C003C00u;
-#pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                __half2 accA[8], accB[8];        // accA[t] = weights (byte 0, byte 2) at bit t; accB: (byte 1, byte 3)
-#pragma unroll
-                for (int t = 0; t < 8; ++t) { accA[t] = z2; accB[t] = z2; }
+                float zhat = use_offset ? sc[Q] : 0.f;
+                __half2 sneg[Q];
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
-                    const uint32_t wv = (wi == 0) ? vec[j].x : (wi == 1) ? vec[j].y : (wi == 2) ? vec[j].z : vec[j].w;
+                    const float sj = use_planes ? sc[j] : 0.f;
+                    zhat += 0.5f * sj;
+                    sneg[j] = __float2half2_rn(-0.5f * sj);               // exact halving of an fp16 value
+                }
+                const __half2 z2 = __float2half2_rn(zhat);
+                const uint8_t* tlane = sT + (lane & 7) * 16;
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        // bits t and t+16 (bytes 0, 2) / t+8 and t+24 (bytes 1, 3) moved to the fp16 sign positions of 1.0
-                        const uint32_t xa = ((wv << (15 - t)) & kSign) | kOne;
-                        const uint32_t xb = ((wv << (7 - t)) & kSign) | kOne;
-                        accA[t] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&xa), accA[t]);
-                        accB[t] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&xb), accB[t]);
+                for (int bi = 0; bi < NB; ++bi) {
+                    __half2 acc[4] = {z2, z2, z2, z2};
+#pragma unroll
+                    for (int j = 0; j < Q; ++j) {
+                        uint32_t wv;
+                        if (WPP == 1) {
+                            wv = (bi < 4) ? vec[j].x : (bi < 8) ? vec[j].y : (bi < 12) ? vec[j].z : vec[j].w;
+                        } else {
+                            const uint32_t w_lo = (bi < 4) ? vec[j].x : vec[j].y, w_hi = (bi < 4) ? vec[j].z : vec[j].w;
+                            wv = bsel ? w_hi : w_lo;
+                        }
+                        const uint32_t byte = (wv >> (8 * (bi & 3))) & 0xffu;
+                        const uint4 sg = *reinterpret_cast<const uint4*>(tlane + byte * 128u);
+                        acc[0] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.x), acc[0]);
+                        acc[1] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.y), acc[1]);
+                        acc[2] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.z), acc[2]);
+                        acc[3] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.w), acc[3]);
                     }
+                    const int ii = bsel * NB + bi;
+                    const int cc = (l + ii) & 15;                         // byte -> 16-byte column (G = 128 rotation)
+                    *reinterpret_cast<uint4*>(sW + row_off + (uint32_t)cc * 128u) =
+                        make_uint4(*reinterpret_cast<const uint32_t*>(&acc[0]), *reinterpret_cast<const uint32_t*>(&acc[1]),
+                                   *reinterpret_cast<const uint32_t*>(&acc[2]), *reinterpret_cast<const uint32_t*>(&acc[3]));
                 }
-                // regroup: a core-matrix row = the 8 weights of one byte (t = 0..7)
+            } else {
+                // rows beyond N (or nothing to contribute): zero rows
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const __half2* src = (b & 1) ? accB : accA;
-                    const uint32_t sel = (b & 2) ? 0x7632u : 0x5410u;          // high or low halves
-                    uint4 out;
-                    out.x = __byte_perm(*reinterpret_cast<const uint32_t*>(&src[0]), *reinterpret_cast<const uint32_t*>(&src[1]), sel);
-                    out.y = __byte_perm(*reinterpret_cast<const uint32_t*>(&src[2]), *reinterpret_cast<const uint32_t*>(&src[3]), sel);
-                    out.z = __byte_perm(*reinterpret_cast<const uint32_t*>(&src[4]), *reinterpret_cast<const uint32_t*>(&src[5]), sel);
-                    out.w = __byte_perm(*reinterpret_cast<const uint32_t*>(&src[6]), *reinterpret_cast<const uint32_t*>(&src[7]), sel);
-                    const int ii = 4 * wi + b;                                  // step -> byte column (G = 128 rotation)
-                    const int cc = 16 * h + ((l + ii) & 15);
-                    *reinterpret_cast<uint4*>(sA + a_row_off + (uint32_t)cc * 128u) = out;
-                }
+                for (int bi = 0; bi < NB; ++bi)
+                    *reinterpret_cast<uint4*>(sW + row_off + (uint32_t)((l + bsel * NB + bi) & 15) * 128u) = make_uint4(0, 0, 0, 0);
             }
-        } else {
-            // rows beyond N (or nothing to contribute): zero rows
-#pragma unroll
-            for (int ii = 0; ii < 16; ++ii)
-                *reinterpret_cast<uint4*>(sA + a_row_off + (uint32_t)(16 * h + ((l + ii) & 15)) * 128u) = make_uint4(0, 0, 0, 0);
         }
 
-        // ---- B: activation tile, tokens m0 .. m0+NT-1, columns step*256 .. +255 -----------------------
-        {
-            const int k_base = step * kStepK;
-#pragma unroll 4
-            for (int idx = tid; idx < NT * 32; idx += kMmaThreads) {
-                const int tok = idx >> 5, c = idx & 31;
-                const int m = m0 + tok, k = k_base + c * 8;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (m < a.M && k < a.K) v = *reinterpret_cast<const uint4*>(a.X + (size_t)m * a.K + k);
-                *reinterpret_cast<uint4*>(sB + (uint32_t)((tok >> 3) * 32 + c) * 128u + (uint32_t)(tok & 7) * 16u) = v;
-            }
-        }
+        // request the next step's weights, then wait for this step's activation tile (all but the newest group)
+        if (step + 1 < step1) load_weights(step + 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
 
-        // ---- MMA: 16 K = 16 slices, issued by one thread; completion arrives on the barrier -------------
-        if (tid == 0) {
+        // ---- MMA: 128 K = 8 slices per token tile, issued by one thread; completion arrives on the barrier ----
+        if (tid == 0 && !(dbg & 4)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (int kk = 0; kk < kStepK / 16; ++kk) {
-                const uint64_t da = make_desc(a_addr + kk * 256), db = make_desc(b_addr + kk * 256);
-                const uint32_t accumulate = (step != step0 || kk != 0) ? 1u : 0u;
-                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-                             :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+            for (int tt = 0; tt < TT; ++tt) {
+#pragma unroll
+                for (int kk = 0; kk < kStepK / 16; ++kk) {
+                    const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + tt * kXTileBytes +
+                                                        (kk >> 2) * (kTileM * 128) + (kk & 3) * 32);
+                    const uint64_t db = desc_noswizzle(w_addr + kk * 256);
+                    const uint32_t accumulate = (step != step0 || kk != 0) ? 1u : 0u;
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                                 : "memory");
+                }
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                          :: "r"(bar_addr) : "memory");
         }
-        // everybody waits for the tensor core to finish reading the tiles before they are overwritten
-        ok = mbar_wait(bar_addr, phase);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (ok && step1 > step0 && !(dbg & 4)) {             // the last step's MMAs
+        ok = __syncthreads_and(mbar_wait(bar_addr, phase) ? 1 : 0) != 0;
         phase ^= 1u;
     }
     if (!ok && a.counters != nullptr && lane == 0) atomicExch(a.counters, 0x7C05u);   // status word: wait ran out
 
-    // ---- epilogue: TMEM -> registers -> Y or partials ---------------------------------------------
+    // ---- epilogue: TMEM (lane = token, column = weight row) -> registers -> Y or partials ---------------
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok && step1 > step0) {
         const int lane_grp = warp & 3, col_half = warp >> 2;            // TMEM lanes 32*lane_grp.., half of the columns
-        const int n = n_tile * kTileN + lane_grp * 32 + lane;
         const size_t n_pad = (size_t)a.n_rb * kTileRows;
+        const bool y_vec_ok = !(a.flags & (ELUTQ_FLAG_OUT_F32 | ELUTQ_FLAG_ACCUMULATE)) && (a.N % 8 == 0) &&
+                              ((reinterpret_cast<uintptr_t>(a.Y) & 15) == 0);
 #pragma unroll 1
-        for (int c0 = col_half * (NT / 2); c0 < (col_half + 1) * (NT / 2); c0 += 32) {
-            uint32_t r[32];
-            const uint32_t taddr = tmem_d + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)c0;
-            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                         : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (n < a.N) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int m = m0 + c0 + i;
-                    if (m < a.M) {
-                        const float v = __uint_as_float(r[i]);
-                        if (splits == 1) store_out(a, (size_t)m * a.N + n, v);
-                        else a.partials[((size_t)split * a.M + m) * n_pad + n] = v;
-                    }
-                }
+        for (int tt = 0; tt < TT; ++tt) {
+            const int m = m0 + tt * kTileM + lane_grp * 32 + lane;
+#pragma unroll 1
+            for (int c0 = col_half * (NW / 2); c0 < (col_half + 1) * (NW / 2); c0 += 32) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_d + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(tt * NW + c0);
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                             : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                               "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                               "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                               "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                             : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (m < a.M) store_row32(a, m, n_tile * NW + c0, r, splits, split, n_pad, y_vec_ok);
             }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"((uint32_t)NT) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"((uint32_t)(TT * NW)) : "memory");
 }
 
-template <int Q, int NT>
-int launch_mma_nt(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    constexpr int kSmem = kABytes + NT * kStepK * 2 + 64;
+template <int Q, int NW, int TT>
+int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
+    constexpr int kSmem = kXStages * TT * kXTileBytes + NW * kStepK * 2 + kSignTableBytes + 64;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(hlq_mma_kernel<Q, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        cudaError_t e = cudaFuncSetAttribute(hlq_mma_kernel<Q, NW, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
     }
-    const int n_tiles = (a.N + kTileN - 1) / kTileN, m_tiles = (a.M + NT - 1) / NT;
-    // K split only while the tile count leaves SMs idle (partials cost M*N*4 bytes per split)
+    const int n_tiles = (a.N + NW - 1) / NW, m_tiles = (a.M + TT * kTileM - 1) / (TT * kTileM);
+    // K split only while the tile count leaves SMs idle (partials cost M*N*4 bytes per split); the partial
+    // buffer holds 2 * n_kc slices.
+    const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;
     int splits = 1;
-    const int n_steps = 2 * a.n_kc;
-    while (splits * 2 <= n_steps && (long long)n_tiles * m_tiles * splits * 2 <= 2LL * num_sms && splits < 16) splits *= 2;
+    while (splits * 2 <= max_splits && (long long)n_tiles * m_tiles * splits * 2 <= (long long)num_sms) splits *= 2;
     if (debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0) splits = debug_env("ELUTQ_DEBUG_MMA_SPLITS");
-    if (splits > n_steps) splits = n_steps;
+    if (splits > max_splits) splits = max_splits;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_tiles, (unsigned)m_tiles, (unsigned)splits);
     cfg.blockDim = dim3(kMmaThreads);
@@ -279,7 +385,8 @@ int launch_mma_nt(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NT>, a, splits);
+    const int dbg = debug_env("ELUTQ_DEBUG_MMA_SKIP") > 0 ? debug_env("ELUTQ_DEBUG_MMA_SKIP") : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT>, a, splits, dbg);
     count_launch(1);
     if (e != cudaSuccess || splits == 1) return (int)e;
     return launch_finalize(a, splits, cfg.numAttrs != 0, stream);
@@ -287,9 +394,17 @@ int launch_mma_nt(const GemmArgs& a, int num_sms, cudaStream_t stream) {
 
 template <int Q>
 int launch_mma_q(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    if (a.M <= 64) return launch_mma_nt<Q, 64>(a, num_sms, stream);
-    if (a.M <= 128) return launch_mma_nt<Q, 128>(a, num_sms, stream);
-    return launch_mma_nt<Q, 256>(a, num_sms, stream);
+    // Two token tiles per CTA once M exceeds one tile; 256 weight rows per CTA unless even the largest K split
+    // would leave most SMs without work.
+    const bool two = a.M > kTileM && debug_env("ELUTQ_DEBUG_MMA_TT") != 1;
+    const long long m_tiles = two ? (a.M + 2 * kTileM - 1) / (2 * kTileM) : (a.M + kTileM - 1) / kTileM;
+    const long long tiles256 = (long long)((a.N + 255) / 256) * m_tiles;
+    const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;
+    bool narrow = tiles256 * max_splits * 2 <= num_sms;
+    if (debug_env("ELUTQ_DEBUG_MMA_NW") == 128) narrow = true;
+    if (debug_env("ELUTQ_DEBUG_MMA_NW") == 256) narrow = false;
+    if (two) return narrow ? launch_mma_cfg<Q, 128, 2>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 2>(a, num_sms, stream);
+    return narrow ? launch_mma_cfg<Q, 128, 1>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 1>(a, num_sms, stream);
 }
 
 }  // namespace
