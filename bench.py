@@ -39,6 +39,7 @@ from workloads import synth  # noqa: E402
 
 METRIC = "HLQ LUT-GEMM achieved HBM GB/s at M=1, 8B shapes (us/call alongside)"
 UNIT = "GB/s"
+FALLBACK_TENSOR_TFLOPS = 1400.0
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -81,6 +82,15 @@ def _peaks():
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback (earlier pool measurement, MEASURED_PEAKS.json absent)"
+
+
+def _tensor_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained, cuBLAS)"
+    except Exception:
+        return FALLBACK_TENSOR_TFLOPS, "fallback (earlier pool measurement, sustained, MEASURED_PEAKS.json absent)"
 
 
 def _traffic_note():
@@ -269,10 +279,21 @@ def run_cuda(args) -> None:
     step_bytes = _bytes_of(calls)
     working_set = sum(l["packed"].numel() for l in layers)
 
+    if args.flags:
+        # variant runs go through the caller-workspace entry point, one workspace per call
+        for l in layers:
+            c = l["call"]
+            l["ws"] = torch.empty(elutq.elutq_workspace_bytes(c.M, c.N, c.K), dtype=torch.uint8, device="cuda")
+            elutq.elutq_workspace_init(l["ws"])
+        torch.cuda.synchronize()
+
     def step():
         for l in layers:
             c = l["call"]
-            elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
+            if args.flags:
+                elutq.elutq_lut_gemm_ws(l["X"], l["packed"], l["Y"], c.M, c.N, c.K, args.flags, l["ws"])
+            else:
+                elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
 
     def step_host():
         for l in layers:
@@ -386,7 +407,20 @@ def run_cuda(args) -> None:
     e2e_value = aggregate_value(step_bytes, world, ms_host / e2e_steps)
     peak, peak_src = _peaks()
     per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
-    traffic = _traffic_note()
+    traffic = _traffic_note() if args.workload == "cfg1" and not args.flags else None
+    roofline = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
+                "peak_source": peak_src,
+                "traffic": traffic.get("dram_bytes_per_step") if traffic else None,
+                "traffic_note": traffic.get("note") if traffic else None}
+    tensor_path = all(c.M >= 64 and c.G == 128 for c in calls) and not (args.flags & 0xF0)
+    if tensor_path:
+        # every call of the step is a dense contraction on the tensor cores: report FLOP/s against the measured
+        # GEMM peak (the sustained figure, since the kernels are timed inside a long step)
+        tpeak, tsrc = _tensor_peak()
+        tf = sum(2.0 * c.M * c.N * c.K for c in calls) / (ms_per_step * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
+                    "peak_source": tsrc, "traffic": None,
+                    "traffic_note": "fp16 operands, fp32 accumulation; fp16 and bf16 share one tensor-core rate"}
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload -------------------------
     cpu = None
@@ -408,10 +442,7 @@ def run_cuda(args) -> None:
                          else "working set fits L2 (L2-hot number, not an HBM figure)",
                    "launch": "CUDA graph of C-ABI calls, programmatic dependent launch" if graph is not None else "stream of C-ABI calls",
                    "parallelism": "replicas only (independent batch per rank, no collective)"},
-        "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
-                     "peak_source": peak_src,
-                     "traffic": traffic.get("dram_bytes_per_step") if traffic else None,
-                     "traffic_note": traffic.get("note") if traffic else None},
+        "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(2 * c.M * c.K for c in calls),
                 "d2h_bytes_per_step": sum(2 * c.M * c.N for c in calls)},
@@ -433,6 +464,8 @@ def main() -> None:
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg1",
                     help="one of %s, or custom:q:N:K[:M],... (G = 128)" % ", ".join(sorted(WORKLOAD_NAMES)))
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0,
+                    help="ELUTQ_FLAG_* bits for every call (kernel-variant comparisons; 0 = the default path)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-call", action="store_true")

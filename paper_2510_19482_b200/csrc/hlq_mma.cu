@@ -47,9 +47,9 @@ constexpr int kSignTableBytes = 256 * 128;   // 256 byte values x 8 bank-group r
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // Shared-memory matrix descriptors (version 1).  Addresses and offsets are in 16-byte units.
-// K-major, no swizzle: leading (K direction) offset 128 bytes, stride (row group) offset 2048 bytes.
+// K-major, no swizzle: leading (K direction) offset 128 bytes, stride (row group) offset 1024 bytes.
 __device__ __forceinline__ uint64_t desc_noswizzle(uint32_t saddr) {
-    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(128u >> 4) << 16) | ((uint64_t)(2048u >> 4) << 32) |
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(128u >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
            ((uint64_t)1 << 46);
 }
 // K-major, 128-byte swizzle: rows of 128 bytes, row groups of 1024 bytes; the leading offset is not used.
@@ -110,15 +110,16 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     constexpr int TILE_BYTES = PLANE_BYTES + 128 * (Q + 1);
     constexpr int PAIRS = NW / 32;                       // item pairs per step: 8 or 4
     constexpr int WPP = (kMmaThreads / 32) / PAIRS;      // warps sharing one item pair: 1 or 2
-    constexpr int NB = 16 / WPP;                         // plane bytes per lane and step
+    constexpr int NB = 8 / WPP;                          // plane bytes per lane and half step
+    constexpr int W_HALF_BYTES = NW * 64 * 2;            // one half (64 k) of the weight tile
     constexpr int X_STAGE_BYTES = TT * kXTileBytes;
     constexpr int W_BYTES = NW * kStepK * 2;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sX = smem;                                  // A operand stages
     uint8_t* sW = smem + kXStages * X_STAGE_BYTES;       // B operand
     uint8_t* sT = sW + W_BYTES;                          // sign table
-    uint64_t* mbar = reinterpret_cast<uint64_t*>(sT + kSignTableBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 1);
+    uint64_t* mbar = reinterpret_cast<uint64_t*>(sT + kSignTableBytes);      // [2]: one per weight-tile half
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int l = lane & 15;
@@ -138,6 +139,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar)) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar + 1)) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // Sign table: entry b holds, for the 8 bits of a plane byte, fp16 +1.0 (bit clear) or -1.0 (bit set),
@@ -207,121 +209,150 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         }
     };
 
-    uint32_t phase = 0;
+    // The packed layout rotates a lane's 16 plane bytes (byte i covers 16-byte column (l + i) mod 16 of the
+    // super-group, which keeps the look-up kernels free of bank conflicts).  Here the halves of the weight tile
+    // are fixed k ranges, so each vector is rotated left by l bytes once per step: byte c then covers column c.
+    auto unrotate = [&]() {
+        const int ws = l >> 2, sh = (l & 3) * 8;
+#pragma unroll
+        for (int j = 0; j < Q; ++j) {
+            const uint32_t v0 = vec[j].x, v1 = vec[j].y, v2 = vec[j].z, v3 = vec[j].w;
+            const uint32_t a0 = (ws & 1) ? v3 : v0, a1 = (ws & 1) ? v0 : v1, a2 = (ws & 1) ? v1 : v2, a3 = (ws & 1) ? v2 : v3;
+            const uint32_t t0 = (ws & 2) ? a2 : a0, t1 = (ws & 2) ? a3 : a1, t2 = (ws & 2) ? a0 : a2, t3 = (ws & 2) ? a1 : a3;
+            vec[j].x = __funnelshift_l(t3, t0, sh);
+            vec[j].y = __funnelshift_l(t0, t1, sh);
+            vec[j].z = __funnelshift_l(t1, t2, sh);
+            vec[j].w = __funnelshift_l(t2, t3, sh);
+        }
+    };
+
+    // One thread's view of a completion barrier: every thread polls for itself; a thread whose wait runs out
+    // raises the status word once and stops waiting, but keeps taking part in every CTA-wide barrier.
     bool ok = true;
+    auto wait_mma = [&](int which, uint32_t parity) {
+        if (!ok || (dbg & 4)) return;
+        if (!mbar_wait(bar_addr + 8u * which, parity)) {
+            ok = false;
+            if (a.counters != nullptr) atomicExch(a.counters, 0x7C05u);
+        }
+    };
+
+    // Dequantise half hb (64 k) of this lane's row into weight buffer hb (BCQ form, sign table).
+    auto dequant_half = [&](int step, int hb) {
+        if (dbg & 2) return;
+        const int u = (step & 3) >> 1;
+        uint8_t* buf = sW + hb * W_HALF_BYTES;
+        const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 8) * 128u + (uint32_t)(l & 7) * 16u;
+        if (rb < a.n_rb && (use_planes | use_offset)) {
+            // parameter record of this super-group: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
+            float sc[Q + 1];
+#pragma unroll
+            for (int c = 0; c <= Q; ++c) {
+                float lo_v = 0.f, hi_v = 0.f;
+#pragma unroll
+                for (int uu = 0; uu < 2; ++uu) {
+                    const int e = uu * (Q + 1) + c;
+                    const uint32_t wv = pw[e >> 1];
+                    const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
+                    if (uu == 0) lo_v = f; else hi_v = f;
+                }
+                sc[c] = u ? hi_v : lo_v;
+            }
+            float zhat = use_offset ? sc[Q] : 0.f;
+            __half2 sneg[Q];
+#pragma unroll
+            for (int j = 0; j < Q; ++j) {
+                const float sj = use_planes ? sc[j] : 0.f;
+                zhat += 0.5f * sj;
+                sneg[j] = __float2half2_rn(-0.5f * sj);               // exact halving of an fp16 value
+            }
+            const __half2 z2 = __float2half2_rn(zhat);
+            const uint8_t* tlane = sT + (lane & 7) * 16;
+#pragma unroll
+            for (int bi = 0; bi < NB; ++bi) {
+                __half2 acc[4] = {z2, z2, z2, z2};
+#pragma unroll
+                for (int j = 0; j < Q; ++j) {
+                    const uint32_t w0 = hb ? vec[j].z : vec[j].x, w1 = hb ? vec[j].w : vec[j].y;
+                    const uint32_t wv = (WPP == 1) ? ((bi < 4) ? w0 : w1) : (bsel ? w1 : w0);
+                    const uint32_t byte = (wv >> (8 * (bi & 3))) & 0xffu;
+                    const uint4 sg = *reinterpret_cast<const uint4*>(tlane + byte * 128u);
+                    acc[0] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.x), acc[0]);
+                    acc[1] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.y), acc[1]);
+                    acc[2] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.z), acc[2]);
+                    acc[3] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.w), acc[3]);
+                }
+                const int cc = bsel * NB + bi;                          // 16-byte column inside the half (0..7)
+                *reinterpret_cast<uint4*>(buf + row_off + (uint32_t)cc * 128u) =
+                    make_uint4(*reinterpret_cast<const uint32_t*>(&acc[0]), *reinterpret_cast<const uint32_t*>(&acc[1]),
+                               *reinterpret_cast<const uint32_t*>(&acc[2]), *reinterpret_cast<const uint32_t*>(&acc[3]));
+            }
+        } else {
+            // rows beyond N (or nothing to contribute): zero rows
+#pragma unroll
+            for (int bi = 0; bi < NB; ++bi)
+                *reinterpret_cast<uint4*>(buf + row_off + (uint32_t)(bsel * NB + bi) * 128u) = make_uint4(0, 0, 0, 0);
+        }
+    };
+
+    // MMAs of one half step (64 k = 4 slices per token tile), issued by one thread; completion arrives on barrier hb.
+    auto issue_mma = [&](int step, int stage, int hb) {
+        if (tid != 0 || (dbg & 4)) return;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+        for (int tt = 0; tt < TT; ++tt) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + tt * kXTileBytes + hb * (kTileM * 128) + kk * 32);
+                const uint64_t db = desc_noswizzle(w_addr + hb * W_HALF_BYTES + kk * 256);
+                const uint32_t accumulate = (step != step0 || hb != 0 || kk != 0) ? 1u : 0u;
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                             :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                             : "memory");
+            }
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     :: "r"(bar_addr + 8u * hb) : "memory");
+    };
+    auto publish = [&]() {     // generic-proxy writes of this thread -> visible to the tensor core, then CTA barrier
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+    };
+
     if (step0 < step1) {
         copy_x(step0, 0);
         load_weights(step0);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 
-    for (int step = step0; step < step1 && ok; ++step) {
+    // Steady state: the tensor core works on one half of the weight tile while the threads dequantise the other.
+    uint32_t phase = 0;                                   // both barriers complete once per step
+    for (int step = step0; step < step1; ++step) {
         const int stage = (step - step0) & 1;
-        if (step > step0 && !(dbg & 4)) {
-            // the tensor core must be done with the weight tile and with the other activation stage
-            ok = __syncthreads_and(mbar_wait(bar_addr, phase) ? 1 : 0) != 0;   // one decision for the whole CTA
-            phase ^= 1u;
-            if (!ok) break;
-        }
+        if (step > step0) wait_mma(0, phase ^ 1u);        // half 0 of the previous step has been read
+        unrotate();
+        dequant_half(step, 0);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");          // this step's activation tile has landed
+        publish();
+        issue_mma(step, stage, 0);
+
+        if (step > step0) wait_mma(1, phase ^ 1u);        // half 1 and the other activation stage have been read
         if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
         asm volatile("cp.async.commit_group;" ::: "memory");
-
-        // ---- B operand: dequantise this lane's row of the step's super-group into the core-matrix layout ----
-        if (!(dbg & 2)) {
-            const int u = (step & 3) >> 1;
-            const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 16) * 128u + (uint32_t)(l & 7) * 16u;
-            if (rb < a.n_rb && (use_planes | use_offset)) {
-                // parameter record of this super-group: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
-                float sc[Q + 1];
-#pragma unroll
-                for (int c = 0; c <= Q; ++c) {
-                    float lo_v = 0.f, hi_v = 0.f;
-#pragma unroll
-                    for (int uu = 0; uu < 2; ++uu) {
-                        const int e = uu * (Q + 1) + c;
-                        const uint32_t wv = pw[e >> 1];
-                        const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
-                        if (uu == 0) lo_v = f; else hi_v = f;
-                    }
-                    sc[c] = u ? hi_v : lo_v;
-                }
-                float zhat = use_offset ? sc[Q] : 0.f;
-                __half2 sneg[Q];
-#pragma unroll
-                for (int j = 0; j < Q; ++j) {
-                    const float sj = use_planes ? sc[j] : 0.f;
-                    zhat += 0.5f * sj;
-                    sneg[j] = __float2half2_rn(-0.5f * sj);               // exact halving of an fp16 value
-                }
-                const __half2 z2 = __float2half2_rn(zhat);
-                const uint8_t* tlane = sT + (lane & 7) * 16;
-#pragma unroll
-                for (int bi = 0; bi < NB; ++bi) {
-                    __half2 acc[4] = {z2, z2, z2, z2};
-#pragma unroll
-                    for (int j = 0; j < Q; ++j) {
-                        uint32_t wv;
-                        if (WPP == 1) {
-                            wv = (bi < 4) ? vec[j].x : (bi < 8) ? vec[j].y : (bi < 12) ? vec[j].z : vec[j].w;
-                        } else {
-                            const uint32_t w_lo = (bi < 4) ? vec[j].x : vec[j].y, w_hi = (bi < 4) ? vec[j].z : vec[j].w;
-                            wv = bsel ? w_hi : w_lo;
-                        }
-                        const uint32_t byte = (wv >> (8 * (bi & 3))) & 0xffu;
-                        const uint4 sg = *reinterpret_cast<const uint4*>(tlane + byte * 128u);
-                        acc[0] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.x), acc[0]);
-                        acc[1] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.y), acc[1]);
-                        acc[2] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.z), acc[2]);
-                        acc[3] = __hfma2(sneg[j], *reinterpret_cast<const __half2*>(&sg.w), acc[3]);
-                    }
-                    const int ii = bsel * NB + bi;
-                    const int cc = (l + ii) & 15;                         // byte -> 16-byte column (G = 128 rotation)
-                    *reinterpret_cast<uint4*>(sW + row_off + (uint32_t)cc * 128u) =
-                        make_uint4(*reinterpret_cast<const uint32_t*>(&acc[0]), *reinterpret_cast<const uint32_t*>(&acc[1]),
-                                   *reinterpret_cast<const uint32_t*>(&acc[2]), *reinterpret_cast<const uint32_t*>(&acc[3]));
-                }
-            } else {
-                // rows beyond N (or nothing to contribute): zero rows
-#pragma unroll
-                for (int bi = 0; bi < NB; ++bi)
-                    *reinterpret_cast<uint4*>(sW + row_off + (uint32_t)((l + bsel * NB + bi) & 15) * 128u) = make_uint4(0, 0, 0, 0);
-            }
-        }
-
-        // request the next step's weights, then wait for this step's activation tile (all but the newest group)
+        dequant_half(step, 1);
         if (step + 1 < step1) load_weights(step + 1);
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-
-        // ---- MMA: 128 K = 8 slices per token tile, issued by one thread; completion arrives on the barrier ----
-        if (tid == 0 && !(dbg & 4)) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-            for (int tt = 0; tt < TT; ++tt) {
-#pragma unroll
-                for (int kk = 0; kk < kStepK / 16; ++kk) {
-                    const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + tt * kXTileBytes +
-                                                        (kk >> 2) * (kTileM * 128) + (kk & 3) * 32);
-                    const uint64_t db = desc_noswizzle(w_addr + kk * 256);
-                    const uint32_t accumulate = (step != step0 || kk != 0) ? 1u : 0u;
-                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
-                                 : "memory");
-                }
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                         :: "r"(bar_addr) : "memory");
-        }
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (ok && step1 > step0 && !(dbg & 4)) {             // the last step's MMAs
-        ok = __syncthreads_and(mbar_wait(bar_addr, phase) ? 1 : 0) != 0;
+        publish();
+        issue_mma(step, stage, 1);
         phase ^= 1u;
     }
-    if (!ok && a.counters != nullptr && lane == 0) atomicExch(a.counters, 0x7C05u);   // status word: wait ran out
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (step1 > step0) {                                  // the last step's MMAs
+        wait_mma(0, phase ^ 1u);
+        wait_mma(1, phase ^ 1u);
+    }
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;
 
     // ---- epilogue: TMEM (lane = token, column = weight row) -> registers -> Y or partials ---------------
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
