@@ -14,11 +14,12 @@
 //              quarter-warp copies the 8 chunks of one token: four full 32-byte sectors on the global side,
 //              eight different bank groups on the shared side.  Two stages, filled by cp.async one step
 //              ahead of the MMAs that read them.
-//   B operand  W_hat tile, NW x 128 fp16, K-major without swizzle: core matrices of 8 rows x 16 bytes in
-//              [row group][k8] order (leading byte offset 128, stride byte offset 2048).  A warp
-//              dequantises two packed items (32 rows): lane 16*i + l owns row l of item i and the step's
-//              super-group, and every packed byte (8 consecutive k of one row) becomes exactly one 16-byte
-//              core-matrix row.
+//   B operand  W_hat tile, NW x 128 fp16, kept as two halves of 64 k, each K-major without swizzle: core
+//              matrices of 8 rows x 16 bytes in [row group][k8] order (leading byte offset 128, stride byte
+//              offset 1024).  A warp dequantises two packed items (32 rows): lane 16*i + l owns row l of
+//              item i and the step's super-group, and every packed byte (8 consecutive k of one row)
+//              becomes exactly one 16-byte core-matrix row.  Each half has its own completion barrier, so
+//              the tensor core reads one half while the threads rebuild the other.
 //   dequant    the BCQ / mirror form of Appendix D: W_hat = z^ + sum_j (-s_j/2) * (+-1).  The +-1.0 fp16
 //              factors of a plane byte (8 weights) come from a 256-entry shared-memory table, one 16-byte
 //              load per byte and plane, followed by four HFMA2.  z^ = z + (1/2) sum s_j is formed in fp32
@@ -28,8 +29,8 @@
 //              stores) or, with a K split, to the fp32 partial buffer that the shared finalize kernel
 //              reduces in ascending order.
 //
-// Every wait is bounded: if the MMA-completion barrier does not flip within the limit the CTA raises the
-// status word, skips the remaining work, still releases its tensor memory and returns.
+// Every wait is bounded: a thread whose MMA-completion barrier does not flip within the limit raises the
+// status word and stops waiting; it still joins every CTA barrier, and the CTA releases its tensor memory.
 #include "common.cuh"
 
 namespace elutq {
