@@ -14,6 +14,8 @@ lut      the same result through the bit-serial look-up-table procedure of
          Appendix B (tables of 2^g partial sums, look-up, per-group scale),
          and the mirror (+-1) form of Appendix D
 storage  bits-per-weight and model-size accounting (Tables 1 and 3 of the paper)
+fit      Algorithm 1 (alternating bit-pattern selection and least squares) that produces
+         (B, s, z) from unquantised fp16 weights
 layout   reference packer / unpacker for the library's device layout
          (a documented pure function; the paper fixes no device layout, so
          this part is "parity unpinned" by the paper and pinned by round trip,

@@ -13,6 +13,7 @@ from .synth import (  # noqa: F401
     scales,
     offsets,
     outlier_columns,
+    dense_weights,
 )
 from . import shapes  # noqa: F401
 from .shapes import (  # noqa: F401

@@ -133,6 +133,16 @@ def activations(seed: int, tag: str, M: int, K: int, outliers: bool = False) -> 
     return x.astype(np.float16)
 
 
+def dense_weights(seed: int, tag: str, N: int, K: int, std: float = 0.02, heavy_frac: float = 0.002) -> np.ndarray:
+    """Unquantised weights fp16 [N, K] for the parameter fitter: N(0, std) with a fraction of entries
+    scaled by 6 (the heavy tails of trained linear layers, which make uniform grids wasteful)."""
+    w = _normal(seed, tag + "/w", 0, N * K) * std
+    u = _raw(seed, tag + "/w_heavy", 0, N * K)
+    heavy = (u >> np.uint64(40)).astype(np.float64) / float(1 << 24) < heavy_frac
+    w = np.where(heavy, w * 6.0, w)
+    return w.reshape(N, K).astype(np.float16)
+
+
 @dataclass
 class HlqLayer:
     """One synthetic HLQ linear layer (host numpy tensors)."""
