@@ -199,6 +199,24 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
 int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
 
 /*
+ * Algorithm 1 (Section 4.2): alternating optimisation of the HLQ parameters, the offline step that
+ * produces what elutq_pack consumes.  For every group of G consecutive weights of a row: uniform
+ * initialisation (Delta = (max - min) / (2^q - 1), s = [Delta, 2 Delta, ...], z = min), then t_max
+ * rounds of bit-pattern selection (nearest of the 2^q candidates, Eq. 5; ties to the smallest code,
+ * code digit j = b_j) and least squares for (s, z) on the selected bits.  A round whose normal
+ * equations are singular (decided exactly, on the integer bit counts) keeps the previous parameters.
+ * Arithmetic is fp64 in a fixed order, so planes and parameters are reproducible bit for bit.
+ *   W          device fp16 [N][K], finite values
+ *   planes     device uint8 [q][N][K], written 0 / 1 (B of the last round)
+ *   scales     device fp16 [N][K/G][q]; offsets device fp16 [N][K/G] (s, z of the last round)
+ *   err_trace  NULL, or device double [(t_max + 1)][N * K/G]: squared error of every group for the
+ *              uniform initialisation (row 0) and after each round (fp64 parameters)
+ * t_max in [1, 1000] (the paper uses 10).  All buffers are caller-owned; nothing is allocated.
+ */
+int elutq_hlq_fit(const void* W, int q, int G, int N, int K, int t_max, uint8_t* planes, void* scales,
+                  void* offsets, double* err_trace, void* stream);
+
+/*
  * Device-side status of the library-owned scratch of `stream` (synchronises the stream).
  * *status is 0 unless a kernel gave up on a bounded wait (then a non-zero code that stays set
  * until elutq_release_scratch).  Kernels never spin without a limit.

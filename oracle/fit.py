@@ -142,6 +142,8 @@ def fit(W: np.ndarray, q: int, G: int, t_max: int = 10, trace: bool = False):
     Returns (planes uint8 [q, N, K], scales fp16 [N, K/G, q], offsets fp16 [N, K/G]) and, with
     trace=True, also the per-group squared error [t_max + 1, N*K/G]: row 0 for the uniform
     initialisation with its own nearest codes, row t after iteration t (fp64 parameters)."""
+    if t_max < 1:
+        raise ValueError("t_max must be at least 1")
     w = _groups(W, G)
     N, K = W.shape
     g = w.shape[0]

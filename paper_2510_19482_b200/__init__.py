@@ -30,6 +30,7 @@ from .binding import (  # noqa: F401
     elutq_lut_gemm_ws,
     elutq_lut_gemm_host,
     elutq_lut_gemm_static,
+    elutq_hlq_fit,
     elutq_device_status,
     elutq_launch_count,
     elutq_release_scratch,

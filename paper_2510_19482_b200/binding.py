@@ -47,6 +47,7 @@ _SIGNATURES = {
     "elutq_lut_gemm_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p, c_size_t, c_void_p]),
     "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_lut_gemm_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_hlq_fit": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
@@ -173,6 +174,20 @@ def elutq_lut_gemm_static(X, packed, Y, M: int, N: int, K: int, stream=None) -> 
     """elutq_lut_gemm for callers that must not allocate: scratch is a fixed 4 MiB array inside the library."""
     _check(lib().elutq_lut_gemm_static(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, _stream(stream)),
            "elutq_lut_gemm_static")
+
+
+def elutq_hlq_fit(W, q: int, G: int, t_max: int = 10, trace: bool = False, stream=None):
+    """Algorithm 1 on a CUDA fp16 matrix W [N, K] -> (planes uint8 [q,N,K], scales fp16 [N,K/G,q],
+    offsets fp16 [N,K/G]) and, with trace=True, the per-group squared error [t_max+1, N*K/G] (fp64)."""
+    import torch
+    N, K = W.shape
+    planes = torch.empty((q, N, K), dtype=torch.uint8, device=W.device)
+    scales = torch.empty((N, K // G, q), dtype=torch.float16, device=W.device)
+    offsets = torch.empty((N, K // G), dtype=torch.float16, device=W.device)
+    tr = torch.empty((t_max + 1, N * (K // G)), dtype=torch.float64, device=W.device) if trace else None
+    _check(lib().elutq_hlq_fit(_ptr(W), q, G, N, K, t_max, _ptr(planes), _ptr(scales), _ptr(offsets),
+                               _ptr(tr) if trace else None, _stream(stream)), "elutq_hlq_fit")
+    return (planes, scales, offsets, tr) if trace else (planes, scales, offsets)
 
 
 def elutq_device_status(stream=None) -> int:

@@ -8,7 +8,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["api.cu", "pack.cu", "lut_gemv.cu", "lut_gemm.cu", "hlq_mma.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "pack.cu", "lut_gemv.cu", "lut_gemm.cu", "hlq_mma.cu", "hlq_fit.cu", "static_scratch.cu"]
 LIB = os.path.join(HERE, "libelutq.so")
 
 

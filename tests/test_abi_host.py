@@ -64,6 +64,12 @@ def test_pointer_validation_happens_before_any_launch():
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x100, 16, 1 << 20, None) == -1  # unknown flag
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x200, 16, 1 << 20, None) == -1
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x50, 16, 1 << 20, None) == -1       # plain g4 + mirror
+    assert L.elutq_hlq_fit(None, 2, 128, 16, 512, 10, None, None, None, None, None) == -1
+    assert L.elutq_hlq_fit(16, 2, 128, 16, 512, 0, 16, 16, 16, None, None) == -1          # t_max < 1
+    assert L.elutq_hlq_fit(16, 5, 128, 16, 512, 10, 16, 16, 16, None, None) == -2         # q out of range
+    assert L.elutq_hlq_fit(16, 2, 128, 16, 500, 10, 16, 16, 16, None, None) == -2         # K % G != 0
+    assert L.elutq_hlq_fit(17, 2, 128, 16, 512, 10, 16, 16, 16, None, None) == -3         # W not 2-byte aligned
+    assert L.elutq_hlq_fit(16, 2, 128, 16, 512, 10, 16, 16, 16, 4, None) == -3            # trace not 8-byte aligned
     assert L.elutq_workspace_init(None, 16, None) == -1
     assert L.elutq_forget(None) == -1
     assert elutq.elutq_launch_count() == before
