@@ -456,6 +456,54 @@ def run_cuda(args) -> None:
         dist.destroy_process_group()
 
 
+def run_fit(args) -> None:
+    """Offline step before the path: elutq_hlq_fit (Algorithm 1) on one dense fp16 layer, `fit:q:G:N:K`."""
+    import torch
+
+    import paper_2510_19482_b200 as elutq
+
+    q, G, N, K = [int(x) for x in args.workload.split(":")[1:5]]
+    t_max = 10
+    W = torch.from_numpy(synth.dense_weights(0, "bench-fit", N, K).view(np.int16)).cuda().view(torch.float16)
+    for _ in range(args.warmup):
+        out = elutq.elutq_hlq_fit(W, q, G, t_max)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        out = elutq.elutq_hlq_fit(W, q, G, t_max)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import fit as ofit
+        rows = max(1, min(N, (1 << 21) // K))
+        Wh = synth.dense_weights(0, "bench-fit", N, K)[:rows]
+        t0 = time.time()
+        ofit.fit(Wh, q, G, t_max)
+        dt = time.time() - t0
+        cpu = {"value": rows * K / dt / 1e9, "unit": "Gweight/s", "cores": _oracle_threads(), "kind": "oracle",
+               "sample": f"first {rows} rows ({dt:.1f} s)"}
+    del out
+    # fp64 pipe work per group and round: selection (1 + 2 * 2^q per weight), error-free right-hand sides are
+    # integer; the (q+1)^3/3-ish solve is repeated by every lane.  Peak: 64 fp64 lanes per clock per SM.
+    sel = G * (1 + 2 * (1 << q))
+    solve = 32 * sum((q + 1 - c - 1) * (2 * (q + 1 - c - 1) + 3) for c in range(q + 1))
+    ops = (N * K // G) * t_max * (sel + solve)
+    peak = 148 * 64 * 1.965e9
+    line = {"metric": "HLQ Algorithm-1 fit throughput", "value": N * K / (ms * 1e-3) / 1e9, "unit": "Gweight/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"Algorithm 1 on a dense fp16 layer N={N} K={K}, q={q}, G={G}, T_max={t_max}"},
+            "roofline": {"bound": "alu", "achieved": ops / (ms * 1e-3) / 1e12, "peak": peak / 1e12, "unit": "T fp64 lane-op/s",
+                         "frac": ops / (ms * 1e-3) / peak,
+                         "peak_source": "148 SMs x 64 fp64 lanes per clock x 1965 MHz (nominal unit count and clock)",
+                         "traffic": None},
+            "gpu_launches": args.steps, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -463,13 +511,19 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg1",
-                    help="one of %s, or custom:q:N:K[:M],... (G = 128)" % ", ".join(sorted(WORKLOAD_NAMES)))
+                    help="one of %s, custom:q:N:K[:M],... (G = 128), or fit:q:G:N:K (the offline parameter fit)"
+                         % ", ".join(sorted(WORKLOAD_NAMES)))
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0,
                     help="ELUTQ_FLAG_* bits for every call (kernel-variant comparisons; 0 = the default path)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-call", action="store_true")
     args = ap.parse_args()
+    if args.workload.startswith("fit:"):
+        args.steps = args.steps or 5
+        args.warmup = max(args.warmup or 3, 3)
+        run_fit(args)
+        return
     if args.workload not in WORKLOAD_NAMES:
         if not args.workload.startswith("custom:"):
             ap.error("unknown workload")

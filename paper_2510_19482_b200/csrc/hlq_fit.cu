@@ -170,7 +170,10 @@ __global__ void __launch_bounds__(kFitWarps * 32) hlq_fit_kernel(const __half* _
             for (int i = 0; i < NV; ++i)
 #pragma unroll
                 for (int j = 0; j < NV; ++j) m[i][j] = A[i][j];
-            long long prev = 1;
+            // The divisions are exact and the quotients (minors of a Gram matrix of 0/1 vectors of length <= 128)
+            // stay below 128^5 < 2^36, so rounding numerator * (1 / prev) in fp64 (relative error < 2^-50)
+            // returns the exact integer; the numerators stay below 2^57.
+            double inv_prev = 1.0;
 #pragma unroll
             for (int c = 0; c < NV; ++c) {
                 singular = singular || (m[c][c] == 0);
@@ -178,8 +181,9 @@ __global__ void __launch_bounds__(kFitWarps * 32) hlq_fit_kernel(const __half* _
 #pragma unroll
                 for (int i = c + 1; i < NV; ++i)
 #pragma unroll
-                    for (int j = c + 1; j < NV; ++j) m[i][j] = (m[i][j] * piv - m[i][c] * m[c][j]) / prev;
-                prev = piv;
+                    for (int j = c + 1; j < NV; ++j)
+                        m[i][j] = __double2ll_rn(__ll2double_rn(m[i][j] * piv - m[i][c] * m[c][j]) * inv_prev);
+                inv_prev = 1.0 / (double)piv;
             }
         }
 
