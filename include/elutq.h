@@ -65,11 +65,20 @@ typedef enum elutq_status {
                                    indices with the top bit clear and the other half is obtained by
                                    negation; same product up to fp32 rounding                              */
 
-#define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 64: stay on the look-up-table kernels.  Without this flag batches of
-                                     64 rows or more (G = 128) take the dequantise-and-contract path: the
+#define ELUTQ_TENSOR_MIN_M 16     /* smallest batch that takes the tensor-core path (measured crossover: the
+                                     look-up kernels win up to M = 8, the tensor cores from M = 16 on) */
+
+#define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 16: stay on the look-up-table kernels.  Without this flag batches of
+                                     ELUTQ_TENSOR_MIN_M rows or more (G = 128) take the dequantise-and-contract path: the
                                      weight tile is rebuilt in fp16 from the bit-planes (BCQ form of
                                      Appendix D) and contracted on the tensor cores with fp32 accumulation;
                                      its results carry the fp16 rounding of W_hat (about 3e-4 relative)     */
+
+#define ELUTQ_FLAG_TABLE_F16 0x100u /* M >= 2, G = 128: table quantisation of Appendix D, first form - the look-up
+                                      tables hold fp16 entries (formed in fp32, rounded once), so one 16-byte
+                                      load serves 8 activation rows instead of 4; accumulation stays fp32.  A
+                                      lossy variant: each entry carries a 2^-11 relative rounding (about 3e-4
+                                      on Y).  Stays on the look-up kernels at every M; ignored at M = 1          */
 
 #define ELUTQ_HEADER_BYTES 128
 

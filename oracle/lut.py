@@ -73,6 +73,35 @@ def lut_matmul(X, planes, scales, offsets, G: int, g: int = 4) -> np.ndarray:
     return Y
 
 
+def table_f16_lut_matmul(X, planes, scales, offsets, G: int, g: int = 8) -> np.ndarray:
+    """Table quantisation, first form (Appendix D): the tables hold fp16 values.
+
+    Every table entry (an exact sum of g activations) is rounded once to fp16 before it is looked up;
+    look-ups, per-group scale multiply and the offset term are as in lut_matmul, in fp64.  The offset
+    term uses the unrounded group sums.  Returns fp64 [M,N]."""
+    X64 = np.asarray(X, dtype=np.float64)
+    M, K = X64.shape
+    q, N, _ = planes.shape
+    if G % g != 0 or K % G != 0:
+        raise ValueError("need g | G | K")
+    s = np.asarray(scales, dtype=np.float64)
+    z = np.asarray(offsets, dtype=np.float64)
+    idx = plane_indices(planes, g)
+    T = K // g
+    t_ar = np.arange(T)[None, :]
+    Y = np.zeros((M, N), dtype=np.float64)
+    for m in range(M):
+        lut = build_lut(X64[m], g)
+        lut16 = lut.astype(np.float16).astype(np.float64)          # one rounding per entry
+        for j in range(q):
+            looked = lut16[t_ar, idx[j]]
+            acc = looked.reshape(N, K // G, G // g).sum(axis=2)
+            Y[m] += (s[:, :, j] * acc).sum(axis=1)
+        S = lut[:, (1 << g) - 1].reshape(K // G, G // g).sum(axis=1)
+        Y[m] += z @ S
+    return Y
+
+
 def mirror_transform(scales, offsets):
     """(s, z) -> (s^, z^) of Appendix D: s^ = s/2, z^ = z + (1/2) sum_j s_j, in fp64."""
     s = np.asarray(scales, dtype=np.float64)

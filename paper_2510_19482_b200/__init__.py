@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     FLAG_CLUSTER_REDUCE,
     FLAG_MIRROR,
     FLAG_LUT_ONLY,
+    FLAG_TABLE_F16,
     lib,
     library_path,
     elutq_packed_bytes,

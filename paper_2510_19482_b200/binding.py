@@ -17,6 +17,7 @@ FLAG_PLAIN_G4 = 0x10
 FLAG_CLUSTER_REDUCE = 0x20
 FLAG_MIRROR = 0x40
 FLAG_LUT_ONLY = 0x80
+FLAG_TABLE_F16 = 0x100
 
 
 class ElutqError(RuntimeError):

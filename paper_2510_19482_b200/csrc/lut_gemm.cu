@@ -20,15 +20,17 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kHalfK = 256;                        // input columns covered by one table set
 
-template <int Q, int G, int MB>
+// TH = true: half-precision tables (table quantisation of Appendix D, first form): an entry holds MB fp16
+// values, so one 8- or 16-byte load serves 4 or 8 activation rows.
+template <int Q, int G, int MB, bool TH = false>
 struct BCfg {
     static constexpr int W = G / 8;
     static constexpr int NSG = 128 / G;
     static constexpr int NPW = 2 * NSG * (Q + 1) / 2;          // parameter words per lane (both halves)
     static constexpr int PLANE_BYTES = 1024 * Q;
     static constexpr int TILE_BYTES = PLANE_BYTES + 128 * NPW;
-    static constexpr int ENTRY_BYTES = 4 * MB;                 // one table entry: MB floats
-    static constexpr int TABLE_BYTES = 256 * 32 * ENTRY_BYTES; // 64 KiB (MB = 2) or 128 KiB (MB = 4)
+    static constexpr int ENTRY_BYTES = (TH ? 2 : 4) * MB;      // one table entry: MB floats (or halves)
+    static constexpr int TABLE_BYTES = 256 * 32 * ENTRY_BYTES; // 64 KiB (8-byte entries) or 128 KiB (16-byte entries)
     static constexpr int SMEM_BYTES = TABLE_BYTES + (256 / G) * MB * 4 + 64;
 };
 
@@ -117,9 +119,91 @@ __device__ __forceinline__ void build_tables_mb(uint8_t* smem, int table_bytes, 
     }
 }
 
-template <int Q, int G, int MB>
+// Half-precision tables for rows m0 .. m0+MB-1 (MB = 4 or 8): same decomposition as build_tables_mb, four rows
+// at a time; every entry is formed in fp32 and rounded once to fp16.  The activation sums for the offset term
+// stay in fp32.
+template <int G, int MB>
+__device__ __forceinline__ void build_tables_half(uint8_t* smem, int table_bytes, const __half* __restrict__ X,
+                                                  int M, int K, int m0, int kc2, int tid) {
+    constexpr int W = G / 8;
+    constexpr int EB = 2 * MB;                          // entry bytes
+    float* gsum = reinterpret_cast<float*>(smem + table_bytes);   // [256/G groups][MB]
+    const int lane = tid & 31, warp = tid >> 5;
+    const int hi = warp & 15, lh = warp >> 4;
+    const int k0 = kc2 * kHalfK + lane * 8;
+    uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * EB + lane * EB;
+#pragma unroll 1
+    for (int quad = 0; quad < MB / 4; ++quad) {
+        float2 x[2][8];                                 // x[p][i] = (x_i of row m0+4quad+2p, x_i of the next row)
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            float xa[8], xb[8];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int m = m0 + 4 * quad + 2 * p + r;
+                float* dst = r ? xb : xa;
+                if (m < M && k0 < K) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                        dst[2 * i] = f.x;
+                        dst[2 * i + 1] = f.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
+        }
+        float2 A[2][8], Bv[2], e7[2];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
+            A[p][1] = fadd2(A[p][0], x[p][0]);
+            A[p][2] = fadd2(A[p][0], x[p][1]);
+            A[p][3] = fadd2(A[p][1], x[p][1]);
+            A[p][4] = fadd2(A[p][0], x[p][2]);
+            A[p][5] = fadd2(A[p][1], x[p][2]);
+            A[p][6] = fadd2(A[p][2], x[p][2]);
+            A[p][7] = fadd2(A[p][3], x[p][2]);
+            Bv[p] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const float2 ea = fadd2(A[0][t], Bv[0]), eb = fadd2(A[1][t], Bv[1]);
+            const __half2 ha = __floats2half2_rn(ea.x, ea.y), hb = __floats2half2_rn(eb.x, eb.y);
+            *reinterpret_cast<uint2*>(rowp + (size_t)t * 32 * EB + quad * 8) =
+                make_uint2(*reinterpret_cast<const uint32_t*>(&ha), *reinterpret_cast<const uint32_t*>(&hb));
+            if (t == 7) { e7[0] = ea; e7[1] = eb; }
+        }
+        if (warp == 31) {   // entry 255: the column's activation sums; reduce over the W columns of a group
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                float sx = e7[p].x, sy = e7[p].y;
+#pragma unroll
+                for (int off = W / 2; off >= 1; off >>= 1) {
+                    sx += __shfl_xor_sync(0xffffffffu, sx, off);
+                    sy += __shfl_xor_sync(0xffffffffu, sy, off);
+                }
+                if ((lane % W) == 0) {
+                    gsum[(lane / W) * MB + 4 * quad + 2 * p] = sx;
+                    gsum[(lane / W) * MB + 4 * quad + 2 * p + 1] = sy;
+                }
+            }
+        }
+    }
+}
+
+template <int Q, int G, int MB, bool TH>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a) {
-    using C = BCfg<Q, G, MB>;
+    using C = BCfg<Q, G, MB, TH>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const float* gsum = reinterpret_cast<const float*>(smem + C::TABLE_BYTES);
 
@@ -134,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
     const int per_mb = n_kc2 * a.n_rb;                 // items per row batch
     const size_t n_pad = (size_t)a.n_rb * kTileRows;
 
-    // Lane column byte offsets inside a table row (column * 8 bytes; the address is doubled for MB = 4),
+    // Lane column byte offsets inside a table row (column * 8 bytes; the address is doubled for 16-byte entries),
     // three steps per register, the fourth byte stays zero and supplies the upper address bytes.
     uint32_t colp[6];
 #pragma unroll
@@ -161,7 +245,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
         const int m0 = mb * MB;
         const int u = kc2 & 1;
         __syncthreads();
-        build_tables_mb<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
+        if (TH) build_tables_half<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
+        else build_tables_mb<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
         __syncthreads();
 
         // group sums of this lane's groups in this half: group (NSG*h + (a+v) % NSG) of the half
@@ -206,7 +291,19 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
                             const int i = v * C::W + ii;
                             // address byte 0 = lane column, byte 1 = weight byte, bytes 2..3 = 0
                             const uint32_t off = prmt(wd[i >> 2], colp[i / 3], 0x7704 + 0x10 * (i & 3) + (i % 3));
-                            if (MB == 2) {
+                            if (TH) {
+                                uint32_t hw[MB / 2];
+                                if constexpr (MB == 4) {
+                                    const uint2 e = *reinterpret_cast<const uint2*>(smem + off);
+                                    hw[0] = e.x; hw[1] = e.y;
+                                } else if constexpr (MB == 8) {
+                                    const uint4 e = *reinterpret_cast<const uint4*>(smem + 2 * off);
+                                    hw[0] = e.x; hw[1] = e.y; hw[2] = e.z; hw[3] = e.w;
+                                }
+#pragma unroll
+                                for (int p = 0; p < MB / 2; ++p)
+                                    acc[p] = fadd2(acc[p], __half22float2(*reinterpret_cast<const __half2*>(&hw[p])));
+                            } else if (MB == 2) {
                                 const float2 e = *reinterpret_cast<const float2*>(smem + off);
                                 acc[0] = fadd2(acc[0], e);
                             } else {
@@ -243,14 +340,14 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
     }
 }
 
-template <int Q, int G, int MB>
+template <int Q, int G, int MB, bool TH = false>
 int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    using C = BCfg<Q, G, MB>;
+    using C = BCfg<Q, G, MB, TH>;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(lut_gemm_kernel<Q, G, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(lut_gemm_kernel<Q, G, MB, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
     }
@@ -276,7 +373,7 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB>, b);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB, TH>, b);
     count_launch(1);
     if (e != cudaSuccess) return (int)e;
     return launch_finalize(b, 2 * a.n_kc, cfg.numAttrs != 0, stream);
@@ -284,6 +381,12 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
 
 template <int Q, int G>
 int launch_qg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
+    if (a.flags & ELUTQ_FLAG_TABLE_F16) {
+        if constexpr (G == 128)
+            return a.M <= 4 ? launch_mb<Q, G, 4, true>(a, num_sms, stream) : launch_mb<Q, G, 8, true>(a, num_sms, stream);
+        else
+            return (int)cudaErrorNotSupported;
+    }
     return a.M == 2 ? launch_mb<Q, G, 2>(a, num_sms, stream) : launch_mb<Q, G, 4>(a, num_sms, stream);
 }
 

@@ -61,7 +61,6 @@ def test_pointer_validation_happens_before_any_launch():
     assert L.elutq_lut_gemm(16, 16, 16, 0, 16, 512, None) == -1
     assert L.elutq_lut_gemm(8, 16, 16, 1, 16, 512, None) == -3
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x3, 16, 1 << 20, None) == -1   # skip-offset + offset-only
-    assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x100, 16, 1 << 20, None) == -1  # unknown flag
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x200, 16, 1 << 20, None) == -1
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x50, 16, 1 << 20, None) == -1       # plain g4 + mirror
     assert L.elutq_hlq_fit(None, 2, 128, 16, 512, 10, None, None, None, None, None) == -1

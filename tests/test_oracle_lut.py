@@ -68,3 +68,35 @@ def test_mirror_identity_and_antisymmetry():
     # the extreme entries are -(x1+..+x4) and +(x1+..+x4)
     np.testing.assert_allclose(lut.mirror_lookup(half, t, np.zeros_like(t), g), -xs.sum(1), atol=1e-12)
     np.testing.assert_allclose(lut.mirror_lookup(half, t, np.full_like(t, 15), g), xs.sum(1), atol=1e-12)
+
+
+def test_f16_tables_are_exact_when_entries_are_representable():
+    """Small-integer activations: every table entry is an integer below 2048, exactly an fp16 value, so the
+    fp16-table procedure must reproduce the definition (Eq. 3 / Eq. 6) exactly."""
+    rng = np.random.default_rng(8)
+    q, G, N, K, M = 2, 32, 12, 128, 3
+    planes = rng.integers(0, 2, size=(q, N, K)).astype(np.uint8)
+    scales = rng.integers(-4, 5, size=(N, K // G, q)).astype(np.float16)
+    offsets = rng.integers(-3, 4, size=(N, K // G)).astype(np.float16)
+    X = rng.integers(-50, 51, size=(M, K)).astype(np.float16)
+    ref = hlq.matmul(X, planes, scales, offsets, G)
+    assert np.array_equal(lut.table_f16_lut_matmul(X, planes, scales, offsets, G), ref)
+
+
+def test_f16_tables_error_is_one_rounding_per_entry():
+    """General activations: the deviation from the definition is bounded by 2^-11 of the looked-up magnitudes
+    weighted by |s| (one fp16 rounding per entry), and is not zero."""
+    rng = np.random.default_rng(9)
+    q, G, N, K, M = 3, 64, 10, 256, 2
+    planes = rng.integers(0, 2, size=(q, N, K)).astype(np.uint8)
+    scales = np.abs(rng.normal(0, 0.02, size=(N, K // G, q))).astype(np.float16)
+    offsets = rng.normal(0, 0.01, size=(N, K // G)).astype(np.float16)
+    X = rng.normal(0, 1, size=(M, K)).astype(np.float16)
+    ref = hlq.matmul(X, planes, scales, offsets, G)
+    got = lut.table_f16_lut_matmul(X, planes, scales, offsets, G)
+    # bound: sum over planes, groups and slices of |s| * 2^-11 * sum|x| of the slice
+    absx = np.abs(X.astype(np.float64)).reshape(M, K // G, G).sum(axis=2)            # [M, groups]
+    bound = 2.0 ** -11 * np.einsum("mg,ngj->mn", absx, np.abs(scales.astype(np.float64)))
+    assert np.all(np.abs(got - ref) <= bound)
+    assert np.any(got != ref)
+    assert hlq.rel_fro_error(got, ref) < 1e-3

@@ -1,0 +1,52 @@
+"""GPU parity of the quantised-table look-up variants (Appendix D, table quantisation) against the oracle's
+restatement of the same procedure, and their accuracy against the definition."""
+import numpy as np
+import pytest
+
+import paper_2510_19482_b200 as elutq
+import workloads
+from oracle import hlq, lut
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import gemm_f32, pack_layer  # noqa: E402
+
+# (q, N, K, M): both row-batch widths (4 and 8 rows per entry), ragged M / N / K tails, every q, M beyond the
+# tensor-core threshold (the flag keeps the call on the look-up kernels)
+CASES = [(2, 200, 1024, 3), (3, 333, 1536, 4), (2, 64, 512, 7), (4, 48, 2560, 9), (1, 130, 640, 8),
+         (2, 500, 2048, 21), (3, 1000, 4096, 16)]
+
+
+@pytest.mark.parametrize("q,N,K,M", CASES)
+def test_f16_tables_match_the_oracle_procedure(q, N, K, M):
+    G = 128
+    layer = workloads.hlq_layer(40, f"tq/{q}/{N}/{K}", q, G, N, K, signed_scales=(q % 2 == 0))
+    X = synth.activations(40, f"tq/x/{M}/{K}", M, K, outliers=(q == 2))
+    packed = pack_layer(layer)
+    y = gemm_f32(X, packed, N, K, elutq.FLAG_TABLE_F16)
+    assert np.all(np.isfinite(y))
+    same = lut.table_f16_lut_matmul(X, layer.planes, layer.scales, layer.offsets, G, g=8)
+    exact = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    # against the same procedure: the kernel forms an entry in fp32 before the fp16 rounding, so an entry can
+    # differ by one fp16 unit only where the fp32 sum crosses a rounding boundary; everything else is fp32
+    # accumulation noise
+    assert hlq.rel_fro_error(y, same) <= 2e-5
+    # against the definition: one 2^-11 rounding per entry, well inside the benchmark's bar
+    err = hlq.rel_fro_error(y, exact)
+    assert 1e-6 < err <= 1e-3
+
+
+def test_f16_tables_flag_is_ignored_for_single_rows_and_rejected_for_small_groups():
+    layer = workloads.hlq_layer(41, "tq/m1", 2, 128, 64, 512)
+    X = synth.activations(41, "tq/m1/x", 1, 512)
+    packed = pack_layer(layer)
+    a = gemm_f32(X, packed, 64, 512, elutq.FLAG_TABLE_F16)
+    b = gemm_f32(X, packed, 64, 512)
+    assert np.array_equal(a, b)
+    layer32 = workloads.hlq_layer(41, "tq/g32", 2, 32, 64, 512)
+    X4 = synth.activations(41, "tq/g32/x", 4, 512)
+    packed32 = pack_layer(layer32)
+    with pytest.raises(elutq.ElutqError) as e:
+        gemm_f32(X4, packed32, 64, 512, elutq.FLAG_TABLE_F16)
+    assert e.value.status == -5
