@@ -39,7 +39,7 @@ namespace elutq {
 
 namespace {
 
-constexpr int kMmaThreads = 256;
+constexpr int kMmaThreads = 256;               // measured: 512 threads (two warps per item pair) are 4-8 % slower
 constexpr int kTileM = 128;                  // tokens per accumulator (UMMA M)
 constexpr int kStepK = 128;                  // K per step
 constexpr int kXTileBytes = kTileM * kStepK * 2;   // one token tile of one step: 2 blocks of [128 tokens][128 bytes]
@@ -159,6 +159,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     // chunk j = tid % 8): 16 bytes at k = step*128 + kb*64 + 8 j, stored at chunk j ^ (r & 7) of row r.
     auto copy_x = [&](int step, int stage) {
         if (dbg & 1) return;
+        constexpr int RPP = kMmaThreads / 8;            // token rows per pass
         const int j = tid & 7, r0 = tid >> 3;
         const uint32_t dst0 = x_addr + (uint32_t)stage * X_STAGE_BYTES + (uint32_t)r0 * 128u + (uint32_t)((j ^ (r0 & 7)) * 16);
 #pragma unroll
@@ -167,9 +168,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             for (int kb = 0; kb < 2; ++kb) {
                 const int k = step * kStepK + kb * 64 + j * 8;
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    const int m = m0 + tt * kTileM + p * 32 + r0;                 // (r0 + 32 p) & 7 == r0 & 7
-                    const uint32_t dst = dst0 + (uint32_t)(tt * kXTileBytes + kb * (kTileM * 128) + p * 32 * 128);
+                for (int p = 0; p < kTileM / RPP; ++p) {
+                    const int m = m0 + tt * kTileM + p * RPP + r0;                // (r0 + RPP p) & 7 == r0 & 7
+                    const uint32_t dst = dst0 + (uint32_t)(tt * kXTileBytes + kb * (kTileM * 128) + p * RPP * 128);
                     if (k < a.K && m < a.M) {
                         const __half* src = a.X + (size_t)m * a.K + k;
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(src) : "memory");
@@ -264,8 +265,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
 #pragma unroll
                 for (int j = 0; j < Q; ++j) {
                     const uint32_t w0 = hb ? vec[j].z : vec[j].x, w1 = hb ? vec[j].w : vec[j].y;
-                    const uint32_t wv = (WPP == 1) ? ((bi < 4) ? w0 : w1) : (bsel ? w1 : w0);
-                    const uint32_t byte = (wv >> (8 * (bi & 3))) & 0xffu;
+                    const int gb = bsel * NB + bi;                              // byte of the half: 0..7
+                    const uint32_t byte = (((gb & 4) ? w1 : w0) >> (8 * (gb & 3))) & 0xffu;
                     // +-s_j/2 for the byte's 8 weights: one multiply moves bits 2p and 2p+1 to the fp16 sign
                     // positions 15 and 31 (the two shifted copies of an 8-bit value do not overlap), one logic
                     // operation flips the signs of the packed -s_j/2, one packed add accumulates
@@ -351,7 +352,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     // ---- epilogue: TMEM (lane = token, column = weight row) -> registers -> Y or partials ---------------
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok && step1 > step0) {
-        const int lane_grp = warp & 3, col_half = warp >> 2;            // TMEM lanes 32*lane_grp.., half of the columns
+        constexpr int CP = kMmaThreads / 128;                            // warps per TMEM lane group: column parts
+        const int lane_grp = warp & 3, col_half = warp >> 2;            // TMEM lanes 32*lane_grp.., one part of the columns
         const size_t n_pad = (size_t)a.n_rb * kTileRows;
         const bool y_vec_ok = !(a.flags & (ELUTQ_FLAG_OUT_F32 | ELUTQ_FLAG_ACCUMULATE)) && (a.N % 8 == 0) &&
                               ((reinterpret_cast<uintptr_t>(a.Y) & 15) == 0);
@@ -359,7 +361,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         for (int tt = 0; tt < TT; ++tt) {
             const int m = m0 + tt * kTileM + lane_grp * 32 + lane;
 #pragma unroll 1
-            for (int c0 = col_half * (NW / 2); c0 < (col_half + 1) * (NW / 2); c0 += 32) {
+            for (int c0 = col_half * (NW / CP); c0 < (col_half + 1) * (NW / CP); c0 += 32) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_d + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(tt * NW + c0);
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
