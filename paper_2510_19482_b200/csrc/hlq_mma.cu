@@ -43,7 +43,6 @@ constexpr int kMmaThreads = 256;               // measured: 512 threads (two war
 constexpr int kTileM = 128;                  // tokens per accumulator (UMMA M)
 constexpr int kStepK = 128;                  // K per step
 constexpr int kXTileBytes = kTileM * kStepK * 2;   // one token tile of one step: 2 blocks of [128 tokens][128 bytes]
-constexpr int kXStages = 2;
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -116,10 +115,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     constexpr int W_HALF_BYTES = NW * 64 * 2;            // one half (64 k) of the weight tile
     constexpr int X_STAGE_BYTES = TT * kXTileBytes;
     constexpr int W_BYTES = NW * kStepK * 2;
+    constexpr int XS = (TT == 1) ? 3 : 2;                // activation stages
+    constexpr int WB = (TT == 1) ? 2 : 1;                // whole weight tiles (each of two halves)
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sX = smem;                                  // A operand stages
-    uint8_t* sW = smem + kXStages * X_STAGE_BYTES;       // B operand
-    uint64_t* mbar = reinterpret_cast<uint64_t*>(sW + W_BYTES);             // [2]: one per weight-tile half
+    uint8_t* sW = smem + XS * X_STAGE_BYTES;             // B operand
+    uint64_t* mbar = reinterpret_cast<uint64_t*>(sW + WB * W_BYTES);        // [2]: one per weight-tile half (TT = 2)
+                                                                            //      or per weight tile (TT = 1)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -229,10 +231,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     };
 
     // Dequantise half hb (64 k) of this lane's row into weight buffer hb (BCQ form, sign table).
-    auto dequant_half = [&](int step, int hb) {
+    auto dequant_half = [&](int step, int hb, int wt) {
         if (dbg & 2) return;
         const int u = (step & 3) >> 1;
-        uint8_t* buf = sW + hb * W_HALF_BYTES;
+        uint8_t* buf = sW + wt * W_BYTES + hb * W_HALF_BYTES;
         const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 8) * 128u + (uint32_t)(l & 7) * 16u;
         if (rb < a.n_rb && (use_planes | use_offset)) {
             // parameter record of this super-group: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
@@ -316,36 +318,80 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         __syncthreads();
     };
 
-    if (step0 < step1) {
-        copy_x(step0, 0);
-        load_weights(step0);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-
-    // Steady state: the tensor core works on one half of the weight tile while the threads dequantise the other.
-    uint32_t phase = 0;                                   // both barriers complete once per step
-    for (int step = step0; step < step1; ++step) {
-        const int stage = (step - step0) & 1;
-        if (step > step0) wait_mma(0, phase ^ 1u);        // half 0 of the previous step has been read
-        unrotate();
-        dequant_half(step, 0);
-        asm volatile("cp.async.wait_group 0;" ::: "memory");          // this step's activation tile has landed
-        publish();
-        issue_mma(step, stage, 0);
-
-        if (step > step0) wait_mma(1, phase ^ 1u);        // half 1 and the other activation stage have been read
-        if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
+    if constexpr (TT == 1) {
+        // One token tile: the MMAs of a step are short next to its dequantisation, so the whole weight tile is
+        // double-buffered and a step has a single CTA barrier: dequantise tile s into buffer s % 2 (last read by the
+        // MMAs of step s - 2, long finished), publish, issue the MMAs of step s, go on with step s + 1.  Three
+        // activation stages, so the copy for step s + 1 never waits for the MMAs of step s - 1 either.
+        auto issue_step = [&](int step, int stage, int wt) {
+            if (tid != 0 || (dbg & 4)) return;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int kk = 0; kk < kStepK / 16; ++kk) {
+                const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + (kk >> 2) * (kTileM * 128) + (kk & 3) * 32);
+                const uint64_t db = desc_noswizzle(w_addr + wt * W_BYTES + (kk >> 2) * W_HALF_BYTES + (kk & 3) * 256);
+                const uint32_t accumulate = (step != step0 || kk != 0) ? 1u : 0u;
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                             :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                         :: "r"(bar_addr + 8u * wt) : "memory");
+        };
+        if (step0 < step1) {
+            copy_x(step0, 0);
+            load_weights(step0);
+        }
         asm volatile("cp.async.commit_group;" ::: "memory");
-        dequant_half(step, 1);
-        if (step + 1 < step1) load_weights(step + 1);
-        publish();
-        issue_mma(step, stage, 1);
-        phase ^= 1u;
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (step1 > step0) {                                  // the last step's MMAs
-        wait_mma(0, phase ^ 1u);
-        wait_mma(1, phase ^ 1u);
+        for (int step = step0; step < step1; ++step) {
+            const int i = step - step0, wt = i & 1;
+            if (i >= 2) wait_mma(wt, (uint32_t)(((i >> 1) - 1) & 1));      // MMAs of step s - 2: buffer and stage are free
+            if (step + 1 < step1) copy_x(step + 1, (i + 1) % 3);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            unrotate();
+            dequant_half(step, 0, wt);
+            dequant_half(step, 1, wt);
+            if (step + 1 < step1) load_weights(step + 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");          // this step's activation tile has landed
+            publish();
+            issue_step(step, i % 3, wt);
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        const int n = step1 - step0;                                       // the last one or two steps' MMAs
+        if (n >= 2) wait_mma((n - 2) & 1, (uint32_t)((((n - 2) >> 1)) & 1));
+        if (n >= 1) wait_mma((n - 1) & 1, (uint32_t)((((n - 1) >> 1)) & 1));
+    } else {
+        if (step0 < step1) {
+            copy_x(step0, 0);
+            load_weights(step0);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+
+        // Steady state: the tensor core works on one half of the weight tile while the threads dequantise the other.
+        uint32_t phase = 0;                                   // both barriers complete once per step
+        for (int step = step0; step < step1; ++step) {
+            const int stage = (step - step0) & 1;
+            if (step > step0) wait_mma(0, phase ^ 1u);        // half 0 of the previous step has been read
+            unrotate();
+            dequant_half(step, 0, 0);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");          // this step's activation tile has landed
+            publish();
+            issue_mma(step, stage, 0);
+
+            if (step > step0) wait_mma(1, phase ^ 1u);        // half 1 and the other activation stage have been read
+            if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            dequant_half(step, 1, 0);
+            if (step + 1 < step1) load_weights(step + 1);
+            publish();
+            issue_mma(step, stage, 1);
+            phase ^= 1u;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (step1 > step0) {                                  // the last step's MMAs
+            wait_mma(0, phase ^ 1u);
+            wait_mma(1, phase ^ 1u);
+        }
     }
     ok = __syncthreads_and(ok ? 1 : 0) != 0;
 
@@ -385,7 +431,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
 
 template <int Q, int NW, int TT>
 int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    constexpr int kSmem = kXStages * TT * kXTileBytes + NW * kStepK * 2 + 64;
+    constexpr int kSmem = (TT == 1 ? 3 : 2) * TT * kXTileBytes + (TT == 1 ? 2 : 1) * NW * kStepK * 2 + 64;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
