@@ -157,28 +157,42 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NW >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
     const uint32_t x_addr = smem_u32(sX), w_addr = smem_u32(sW), bar_addr = smem_u32(mbar);
 
-    // Asynchronous copy of the activation tile(s) of one step into a stage.  Thread (token r = tid / 8 + 32 p,
-    // chunk j = tid % 8): 16 bytes at k = step*128 + kb*64 + 8 j, stored at chunk j ^ (r & 7) of row r.
+    // Asynchronous copy of the activation tile(s) of one step into a stage.  Thread (token r = tid / 8 + RPP p,
+    // chunk j = tid % 8): 16 bytes at k = step*128 + kb*64 + 8 j, stored at chunk j ^ (r & 7) of row r.  Rows
+    // beyond M and columns beyond K are zero-filled by a copy of source size 0 (its address is clamped to a
+    // valid row, nothing is read), so the loop carries no branches.
+    constexpr int RPP = kMmaThreads / 8;            // token rows per pass
+    constexpr int NPASS = kTileM / RPP;
+    const __half* x_src[TT * NPASS];
+    uint32_t x_live = 0;                            // bit (tt * NPASS + p): the row exists
+    {
+        const int j = tid & 7, r0 = tid >> 3;
+#pragma unroll
+        for (int tt = 0; tt < TT; ++tt)
+#pragma unroll
+            for (int p = 0; p < NPASS; ++p) {
+                const int m = m0 + tt * kTileM + p * RPP + r0;
+                x_src[tt * NPASS + p] = a.X + (size_t)(m < a.M ? m : a.M - 1) * a.K + j * 8;
+                if (m < a.M) x_live |= 1u << (tt * NPASS + p);
+            }
+    }
     auto copy_x = [&](int step, int stage) {
         if (dbg & 1) return;
-        constexpr int RPP = kMmaThreads / 8;            // token rows per pass
         const int j = tid & 7, r0 = tid >> 3;
         const uint32_t dst0 = x_addr + (uint32_t)stage * X_STAGE_BYTES + (uint32_t)r0 * 128u + (uint32_t)((j ^ (r0 & 7)) * 16);
 #pragma unroll
-        for (int tt = 0; tt < TT; ++tt) {
+        for (int kb = 0; kb < 2; ++kb) {
+            const int k = step * kStepK + kb * 64;                     // k + 8 j < K for every j or for none (K % 64 == 0)
+            const uint32_t live = (k < a.K) ? x_live : 0u;
+            const int koff = (k < a.K) ? k : 0;
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb) {
-                const int k = step * kStepK + kb * 64 + j * 8;
+            for (int tt = 0; tt < TT; ++tt) {
 #pragma unroll
-                for (int p = 0; p < kTileM / RPP; ++p) {
-                    const int m = m0 + tt * kTileM + p * RPP + r0;                // (r0 + RPP p) & 7 == r0 & 7
+                for (int p = 0; p < NPASS; ++p) {                       // (r0 + RPP p) & 7 == r0 & 7
                     const uint32_t dst = dst0 + (uint32_t)(tt * kXTileBytes + kb * (kTileM * 128) + p * RPP * 128);
-                    if (k < a.K && m < a.M) {
-                        const __half* src = a.X + (size_t)m * a.K + k;
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(src) : "memory");
-                    } else {
-                        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" :: "r"(dst), "r"(0u) : "memory");
-                    }
+                    const uint32_t nbytes = ((live >> (tt * NPASS + p)) & 1u) ? 16u : 0u;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                                 :: "r"(dst), "l"(x_src[tt * NPASS + p] + koff), "r"(nbytes) : "memory");
                 }
             }
         }
