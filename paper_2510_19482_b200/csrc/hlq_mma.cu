@@ -244,37 +244,42 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         }
     };
 
-    // Dequantise half hb (64 k) of this lane's row into weight buffer hb (BCQ form, sign table).
-    auto dequant_half = [&](int step, int hb, int wt) {
-        if (dbg & 2) return;
+    // Parameters of the step's super-group for this lane's row, decoded once per step: halves
+    // [u*(Q+1) .. u*(Q+1)+Q] of the parameter words = s_0..s_{Q-1}, z.
+    uint32_t sneg[Q];                                              // (-s_j/2, -s_j/2) as packed fp16
+    __half2 z2;                                                    // (z^, z^)
+    auto decode_params = [&](int step) {
         const int u = (step & 3) >> 1;
+        float sc[Q + 1];
+#pragma unroll
+        for (int c = 0; c <= Q; ++c) {
+            float lo_v = 0.f, hi_v = 0.f;
+#pragma unroll
+            for (int uu = 0; uu < 2; ++uu) {
+                const int e = uu * (Q + 1) + c;
+                const uint32_t wv = pw[e >> 1];
+                const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
+                if (uu == 0) lo_v = f; else hi_v = f;
+            }
+            sc[c] = u ? hi_v : lo_v;
+        }
+        float zhat = use_offset ? sc[Q] : 0.f;
+#pragma unroll
+        for (int j = 0; j < Q; ++j) {
+            const float sj = use_planes ? sc[j] : 0.f;
+            zhat += 0.5f * sj;
+            const __half2 h2 = __float2half2_rn(-0.5f * sj);           // exact halving of an fp16 value
+            sneg[j] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
+        z2 = __float2half2_rn(zhat);
+    };
+
+    // Dequantise half hb (64 k) of this lane's row into half hb of weight tile wt (BCQ form, in registers).
+    auto dequant_half = [&](int hb, int wt) {
+        if (dbg & 2) return;
         uint8_t* buf = sW + wt * W_BYTES + hb * W_HALF_BYTES;
         const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 8) * 128u + (uint32_t)(l & 7) * 16u;
         if (rb < a.n_rb && (use_planes | use_offset)) {
-            // parameter record of this super-group: halves [u*(Q+1) .. u*(Q+1)+Q] = s_0..s_{Q-1}, z
-            float sc[Q + 1];
-#pragma unroll
-            for (int c = 0; c <= Q; ++c) {
-                float lo_v = 0.f, hi_v = 0.f;
-#pragma unroll
-                for (int uu = 0; uu < 2; ++uu) {
-                    const int e = uu * (Q + 1) + c;
-                    const uint32_t wv = pw[e >> 1];
-                    const float f = __half2float(__ushort_as_half((unsigned short)((e & 1) ? (wv >> 16) : (wv & 0xffffu))));
-                    if (uu == 0) lo_v = f; else hi_v = f;
-                }
-                sc[c] = u ? hi_v : lo_v;
-            }
-            float zhat = use_offset ? sc[Q] : 0.f;
-            uint32_t sneg[Q];                                          // (-s_j/2, -s_j/2) as packed fp16
-#pragma unroll
-            for (int j = 0; j < Q; ++j) {
-                const float sj = use_planes ? sc[j] : 0.f;
-                zhat += 0.5f * sj;
-                const __half2 h2 = __float2half2_rn(-0.5f * sj);       // exact halving of an fp16 value
-                sneg[j] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-            const __half2 z2 = __float2half2_rn(zhat);
 #pragma unroll
             for (int bi = 0; bi < NB; ++bi) {
                 __half2 acc[4] = {z2, z2, z2, z2};
@@ -363,8 +368,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             if (step + 1 < step1) copy_x(step + 1, (i + 1) % 3);
             asm volatile("cp.async.commit_group;" ::: "memory");
             unrotate();
-            dequant_half(step, 0, wt);
-            dequant_half(step, 1, wt);
+            decode_params(step);
+            dequant_half(0, wt);
+            dequant_half(1, wt);
             if (step + 1 < step1) load_weights(step + 1);
             asm volatile("cp.async.wait_group 1;" ::: "memory");          // this step's activation tile has landed
             publish();
@@ -387,7 +393,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             const int stage = (step - step0) & 1;
             if (step > step0) wait_mma(0, phase ^ 1u);        // half 0 of the previous step has been read
             unrotate();
-            dequant_half(step, 0, 0);
+            decode_params(step);
+            dequant_half(0, 0);
             asm volatile("cp.async.wait_group 0;" ::: "memory");          // this step's activation tile has landed
             publish();
             issue_mma(step, stage, 0);
@@ -395,7 +402,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             if (step > step0) wait_mma(1, phase ^ 1u);        // half 1 and the other activation stage have been read
             if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            dequant_half(step, 1, 0);
+            dequant_half(1, 0);
             if (step + 1 < step1) load_weights(step + 1);
             publish();
             issue_mma(step, stage, 1);
