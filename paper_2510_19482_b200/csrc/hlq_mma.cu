@@ -105,7 +105,7 @@ __device__ __forceinline__ void store_row32(const GemmArgs& a, int m, int n0, co
 
 // NW = weight rows per CTA (UMMA N: 128 or 256); TT = token tiles of 128 per CTA (1 or 2).
 template <int Q, int NW, int TT>
-__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits, const int dbg) {
+__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits) {
     constexpr int NPW = Q + 1;                           // parameter words per lane at G = 128
     constexpr int PLANE_BYTES = 1024 * Q;
     constexpr int TILE_BYTES = PLANE_BYTES + 128 * (Q + 1);
@@ -177,7 +177,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             }
     }
     auto copy_x = [&](int step, int stage) {
-        if (dbg & 1) return;
         const int j = tid & 7, r0 = tid >> 3;
         const uint32_t dst0 = x_addr + (uint32_t)stage * X_STAGE_BYTES + (uint32_t)r0 * 128u + (uint32_t)((j ^ (r0 & 7)) * 16);
 #pragma unroll
@@ -237,7 +236,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     // raises the status word once and stops waiting, but keeps taking part in every CTA-wide barrier.
     bool ok = true;
     auto wait_mma = [&](int which, uint32_t parity) {
-        if (!ok || (dbg & 4)) return;
+        if (!ok) return;
         if (!mbar_wait(bar_addr + 8u * which, parity)) {
             ok = false;
             if (a.counters != nullptr) atomicExch(a.counters, 0x7C05u);
@@ -276,7 +275,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
 
     // Dequantise half hb (64 k) of this lane's row into half hb of weight tile wt (BCQ form, in registers).
     auto dequant_half = [&](int hb, int wt) {
-        if (dbg & 2) return;
         uint8_t* buf = sW + wt * W_BYTES + hb * W_HALF_BYTES;
         const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 8) * 128u + (uint32_t)(l & 7) * 16u;
         if (rb < a.n_rb && (use_planes | use_offset)) {
@@ -313,7 +311,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
 
     // MMAs of one half step (64 k = 4 slices per token tile), issued by one thread; completion arrives on barrier hb.
     auto issue_mma = [&](int step, int stage, int hb) {
-        if (tid != 0 || (dbg & 4)) return;
+        if (tid != 0) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int tt = 0; tt < TT; ++tt) {
@@ -343,7 +341,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         // MMAs of step s - 2, long finished), publish, issue the MMAs of step s, go on with step s + 1.  Three
         // activation stages, so the copy for step s + 1 never waits for the MMAs of step s - 1 either.
         auto issue_step = [&](int step, int stage, int wt) {
-            if (tid != 0 || (dbg & 4)) return;
+            if (tid != 0) return;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int kk = 0; kk < kStepK / 16; ++kk) {
@@ -479,8 +477,7 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
-    const int dbg = debug_env("ELUTQ_DEBUG_MMA_SKIP") > 0 ? debug_env("ELUTQ_DEBUG_MMA_SKIP") : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT>, a, splits, dbg);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT>, a, splits);
     count_launch(1);
     if (e != cudaSuccess || splits == 1) return (int)e;
     return launch_finalize(a, splits, cfg.numAttrs != 0, stream);
