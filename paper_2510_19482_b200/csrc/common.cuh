@@ -76,7 +76,8 @@ int launch_lut_gemv(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t s
 int launch_lut_gemm(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 int launch_hlq_mma(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t stream);
 
-int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream);
+// col0 / cols restrict the reduction to output columns [col0, col0 + cols) (cols = 0: all N columns).
+int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream, int col0 = 0, int cols = 0);
 int debug_env(const char* name);
 void count_launch(unsigned n = 1);
 

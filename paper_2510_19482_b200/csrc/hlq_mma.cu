@@ -105,7 +105,7 @@ __device__ __forceinline__ void store_row32(const GemmArgs& a, int m, int n0, co
 
 // NW = weight rows per CTA (UMMA N: 128 or 256); TT = token tiles of 128 per CTA (1 or 2).
 template <int Q, int NW, int TT>
-__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits) {
+__global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs a, const int splits, const int n_tile0) {
     constexpr int NPW = Q + 1;                           // parameter words per lane at G = 128
     constexpr int PLANE_BYTES = 1024 * Q;
     constexpr int TILE_BYTES = PLANE_BYTES + 128 * (Q + 1);
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int l = lane & 15;
-    const int n_tile = blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
+    const int n_tile = n_tile0 + blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
     const int m0 = m_tile * (TT * kTileM);
     const int n_steps = 4 * a.n_kc;                                   // super-groups
     const int step0 = (int)((long long)n_steps * split / splits);
@@ -460,27 +460,56 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
         configured[dev] = true;
     }
     const int n_tiles = (a.N + NW - 1) / NW, m_tiles = (a.M + TT * kTileM - 1) / (TT * kTileM);
-    // K split only while the tile count leaves SMs idle (partials cost M*N*4 bytes per split); the partial
-    // buffer holds 2 * n_kc slices.
-    const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;
-    int splits = 1;
-    while (splits * 2 <= max_splits && (long long)n_tiles * m_tiles * splits * 2 <= (long long)num_sms) splits *= 2;
-    if (debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0) splits = debug_env("ELUTQ_DEBUG_MMA_SPLITS");
-    if (splits > max_splits) splits = max_splits;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)n_tiles, (unsigned)m_tiles, (unsigned)splits);
-    cfg.blockDim = dim3(kMmaThreads);
-    cfg.dynamicSmemBytes = kSmem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT>, a, splits);
-    count_launch(1);
-    if (e != cudaSuccess || splits == 1) return (int)e;
-    return launch_finalize(a, splits, cfg.numAttrs != 0, stream);
+    const long long tiles = (long long)n_tiles * m_tiles;
+    const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;   // the partial buffer holds 2 * n_kc slices
+    const bool pdl = debug_env("ELUTQ_DEBUG_NO_PDL") == 0;
+
+    auto launch = [&](int n_tile0, int n_count, int splits) -> cudaError_t {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)n_count, (unsigned)m_tiles, (unsigned)splits);
+        cfg.blockDim = dim3(kMmaThreads);
+        cfg.dynamicSmemBytes = kSmem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl ? 1 : 0;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT>, a, splits, n_tile0);
+        count_launch(1);
+        return e;
+    };
+
+    // Fewer tiles than SMs: K split while the tile count leaves SMs idle (partials cost M*N*4 bytes per split).
+    if (tiles <= num_sms || debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0 || debug_env("ELUTQ_DEBUG_MMA_NO_TAIL") > 0) {
+        int splits = 1;
+        while (splits * 2 <= max_splits && tiles * splits * 2 <= (long long)num_sms) splits *= 2;
+        if (debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0) splits = debug_env("ELUTQ_DEBUG_MMA_SPLITS");
+        if (splits > max_splits) splits = max_splits;
+        cudaError_t e = launch(0, n_tiles, splits);
+        if (e != cudaSuccess || splits == 1) return (int)e;
+        return launch_finalize(a, splits, pdl, stream);
+    }
+
+    // More tiles than SMs: whole rounds of whole tiles, then the column stripe that would make a thin last round
+    // is launched on its own with a K split that fills the GPU (reduced by the finalize kernel over those columns).
+    const long long full = tiles / num_sms * num_sms;               // tiles in whole rounds
+    int n_main = (int)(full / m_tiles);                             // whole columns of tiles within them
+    if (n_main > n_tiles) n_main = n_tiles;
+    const long long tail_tiles = (long long)(n_tiles - n_main) * m_tiles;
+    int tail_splits = tail_tiles > 0 ? (int)(num_sms / tail_tiles) : 1;
+    if (tail_splits > max_splits) tail_splits = max_splits;
+    if (tail_splits > 4 * a.n_kc) tail_splits = 4 * a.n_kc;
+    // worth it when the tail round shrinks by more than the extra launch and its partial-sum traffic cost
+    const bool use_tail = tail_tiles > 0 && tail_splits >= 2 && n_main > 0 &&
+                          (tail_tiles + num_sms - 1) / num_sms == 1;
+    if (!use_tail) return (int)launch(0, n_tiles, 1);
+    cudaError_t e = launch(0, n_main, 1);
+    if (e != cudaSuccess) return (int)e;
+    e = launch(n_main, n_tiles - n_main, tail_splits);
+    if (e != cudaSuccess) return (int)e;
+    const int col0 = n_main * NW;
+    return launch_finalize(a, tail_splits, pdl, stream, col0, a.N - col0);
 }
 
 template <int Q>

@@ -403,12 +403,12 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
 // K-split epilogue: Y[m][n] = sum over the K chunks of partials[chunk][m][n], chunks added in ascending
 // order (bit-reproducible), then the output conversion.  One thread per output element.  Launched right
 // behind the main kernel with programmatic dependent launch: the grid dependency wait is the only barrier.
-__global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, const int n_chunks) {
+__global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, const int n_chunks, const int col0, const int cols) {
     grid_launch_dependents();
     grid_dependency_wait();
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= (long long)a.M * a.N) return;
-    const int m = (int)(idx / a.N), row = (int)(idx % a.N);
+    if (idx >= (long long)a.M * cols) return;
+    const int m = (int)(idx / cols), row = col0 + (int)(idx % cols);
     const size_t n_pad = (size_t)a.n_rb * kTileRows;
     store_out(a, (size_t)m * a.N + row, sum_chunks(a.partials + (size_t)m * n_pad + row, (size_t)a.M * n_pad, n_chunks));
 }
@@ -418,14 +418,15 @@ __global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, con
 // of p: a fixed order again, so the result stays bit-reproducible (it differs in rounding from the
 // single-thread order, which is why this form is only used above 8 chunks, where no other reduction
 // path exists to be compared with).
-__global__ void __launch_bounds__(256) lut_finalize_parts_kernel(const GemmArgs a, const int n_chunks, const int per) {
+__global__ void __launch_bounds__(256) lut_finalize_parts_kernel(const GemmArgs a, const int n_chunks, const int per,
+                                                                 const int col0, const int cols) {
     __shared__ float sub[8][32];
     grid_launch_dependents();
     grid_dependency_wait();
     const int lane = threadIdx.x & 31, part = threadIdx.x >> 5, parts = blockDim.x >> 5;
     const long long idx = (long long)blockIdx.x * 32 + lane;
-    const bool live = idx < (long long)a.M * a.N;
-    const int m = live ? (int)(idx / a.N) : 0, row = live ? (int)(idx % a.N) : 0;
+    const bool live = idx < (long long)a.M * cols;
+    const int m = live ? (int)(idx / cols) : 0, row = live ? col0 + (int)(idx % cols) : 0;
     const size_t n_pad = (size_t)a.n_rb * kTileRows;
     const int c0 = part * per, c1 = min(n_chunks, c0 + per);
     float v = 0.f;
@@ -455,7 +456,8 @@ int debug_env(const char* name) {
     return val;
 }
 
-int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream) {
+int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream, int col0, int cols) {
+    if (cols <= 0) { col0 = 0; cols = a.N; }
     cudaLaunchConfig_t cfg = {};
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -463,7 +465,7 @@ int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    const long long outputs = (long long)a.M * a.N;
+    const long long outputs = (long long)a.M * cols;
     // The reduction is latency-bound (n_chunks independent loads per output), so it wants all the
     // parallelism it can get: above 8 chunks, and while the outputs alone do not fill the GPU, several
     // warps share an output's chunks (measured on N = 8192, K = 28672: 8.2 us -> 2.1 us).
@@ -479,12 +481,12 @@ int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stre
         const int per = (n_chunks + parts - 1) / parts;
         cfg.gridDim = dim3((unsigned)((outputs + 31) / 32));
         cfg.blockDim = dim3(32 * parts);
-        e = cudaLaunchKernelEx(&cfg, lut_finalize_parts_kernel, a, n_chunks, per);
+        e = cudaLaunchKernelEx(&cfg, lut_finalize_parts_kernel, a, n_chunks, per, col0, cols);
     } else {
         // one thread per output element
         cfg.gridDim = dim3((unsigned)((outputs + 255) / 256));
         cfg.blockDim = dim3(256);
-        e = cudaLaunchKernelEx(&cfg, lut_finalize_kernel, a, n_chunks);
+        e = cudaLaunchKernelEx(&cfg, lut_finalize_kernel, a, n_chunks, col0, cols);
     }
     count_launch(1);
     return (int)e;

@@ -23,7 +23,8 @@ TOL = 1e-3
 
 # (q, N, K, M): one tile, ragged N / M / K tails, every q, several token tiles, a K split
 CASES = [(2, 512, 1024, 16), (3, 300, 1536, 40), (2, 256, 512, 64), (2, 200, 1024, 100), (3, 1000, 1536, 128), (4, 384, 2560, 300),
-         (1, 130, 640, 65), (2, 4096, 4096, 128), (3, 512, 4096, 700)]
+         (1, 130, 640, 65), (2, 4096, 4096, 128), (3, 512, 4096, 700),
+         (2, 4096, 512, 2560)]      # 160 tiles: whole rounds plus a K-split tail stripe
 
 
 @pytest.mark.parametrize("q,N,K,M", CASES)
