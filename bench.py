@@ -473,11 +473,15 @@ def run_cuda(args) -> None:
     # ---- CPU baseline: the oracle on a bounded sample of the same workload -------------------------
     cpu = None
     if not args.no_cpu_baseline:
-        rows = 1024
+        # a short probe sizes the sample for about 15 s of CPU work (bounded below and above)
+        probe_rows = 256
+        _, probe_dt = _time_oracle(_oracle_sample(calls, probe_rows, seed=0), 1, 0)
+        rows = int(max(256, min(4096, probe_rows * 15.0 / max(probe_dt, 1e-3))))   # generation time bounds it too
         sample = _oracle_sample(calls, rows, seed=0)
         gbs, dt = _time_oracle(sample, 1, 0)
         cpu = {"value": gbs, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
-               "sample": f"first {rows} output rows of each of the {len(calls)} layers, one pass ({dt:.1f} s)"}
+               "sample": f"first {rows} output rows (or all, where a layer has fewer) of each of the {len(calls)} layers, "
+                         f"one pass ({dt:.1f} s)"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
