@@ -389,14 +389,28 @@ def run_cuda(args) -> None:
         ms_median, ms_min = singles[len(singles) // 2], singles[0]
 
         # ---- end to end through the host entry point ---------------------------------------------
+        # (the same launch mode as above: a CUDA graph of the public host-buffer calls, whose copy nodes read the
+        #  pinned inputs and write the pinned outputs on every replay)
         e2e_steps = max(1, min(args.steps, 200))
+        host_graph = None
+        if graph is not None:
+            host_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(host_graph, stream=stream):
+                step_host()
+
+        def run_host():
+            if host_graph is not None:
+                host_graph.replay()
+            else:
+                step_host()
+
         for _ in range(min(args.warmup, 20)):
-            step_host()
+            run_host()
         barrier()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         h0.record()
         for _ in range(e2e_steps):
-            step_host()
+            run_host()
         h1.record()
         barrier()
         ms_host = h0.elapsed_time(h1)
