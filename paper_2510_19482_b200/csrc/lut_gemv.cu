@@ -271,13 +271,30 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         // every consumed vector are refilled with the next item's data.
         auto do_item = [&](auto has_next_c) {
             constexpr bool HAS_NEXT = decltype(has_next_c)::value != 0;
-            float prm[C::GL * (Q + 1)];
+            // Parameters: converted up front (mirror mode rewrites them) or kept as the packed fp16 words and
+            // converted where used, which holds half as many registers through the look-up loop.
+            constexpr bool LAZY = (MODE != kModeMirror) && Q >= 3;
+            float prm[LAZY ? 1 : C::GL * (Q + 1)];
+            uint32_t praw[LAZY ? C::NPW : 1];
+            if constexpr (LAZY) {
 #pragma unroll
-            for (int i = 0; i < C::NPW; ++i) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&buf.p[i]));
-                prm[2 * i] = f.x;
-                prm[2 * i + 1] = f.y;
+                for (int i = 0; i < C::NPW; ++i) praw[i] = buf.p[i];
+            } else {
+#pragma unroll
+                for (int i = 0; i < C::NPW; ++i) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&buf.p[i]));
+                    prm[2 * i] = f.x;
+                    prm[2 * i + 1] = f.y;
+                }
             }
+            auto param = [&](int idx) -> float {          // idx is a constant after unrolling
+                if constexpr (LAZY) {
+                    const __half2 h2 = *reinterpret_cast<const __half2*>(&praw[idx >> 1]);
+                    return (idx & 1) ? __high2float(h2) : __low2float(h2);
+                } else {
+                    return prm[idx];
+                }
+            };
             if (HAS_NEXT) static_for<0, C::NPW>([&](auto i) { buf.p[i] = ldg_stream_u32<i * 128>(npp); });
             if (MODE == kModeMirror) {
                 // s^ = s / 2 and z^ = z + (1/2) sum_j s_j, formed in fp32 (exact halving, one rounding for z^)
@@ -324,14 +341,14 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
                             }
                             acc = fadd2(acc, make_float2(e[0], e[1]));
                         }
-                        y = fmaf(prm[(u * C::NSG + v) * (Q + 1) + j], acc.x + acc.y, y);
+                        y = fmaf(param((u * C::NSG + v) * (Q + 1) + j), acc.x + acc.y, y);
                     }
                     // the vector is dead now: refill its registers with the next item's data
                     if (HAS_NEXT) buf.v[uj] = ldg_stream_v4<uj * 512>(nvp);
                 });
             }
 #pragma unroll
-            for (int gi = 0; gi < C::GL; ++gi) y = fmaf(prm[gi * (Q + 1) + Q], S[gi], y);
+            for (int gi = 0; gi < C::GL; ++gi) y = fmaf(param(gi * (Q + 1) + Q), S[gi], y);
             y += __shfl_xor_sync(0xffffffffu, y, 16);
 
             const int row = (it - kc * a.n_rb) * kTileRows + l;
