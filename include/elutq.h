@@ -65,10 +65,10 @@ typedef enum elutq_status {
                                    indices with the top bit clear and the other half is obtained by
                                    negation; same product up to fp32 rounding                              */
 
-#define ELUTQ_TENSOR_MIN_M 16     /* smallest batch that takes the tensor-core path (measured crossover: the
-                                     look-up kernels win up to M = 8, the tensor cores from M = 16 on) */
+#define ELUTQ_TENSOR_MIN_M 9      /* smallest batch that takes the tensor-core path (measured crossover: the two
+                                     paths are level at M = 8, the tensor cores win from M = 9 on)          */
 
-#define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 16: stay on the look-up-table kernels.  Without this flag batches of
+#define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 9: stay on the look-up-table kernels.  Without this flag batches of
                                      ELUTQ_TENSOR_MIN_M rows or more (G = 128) take the dequantise-and-contract path: the
                                      weight tile is rebuilt in fp16 from the bit-planes (BCQ form of
                                      Appendix D) and contracted on the tensor cores with fp32 accumulation;

@@ -35,7 +35,7 @@ def test_batched_gemm_matches_oracle(q, G, N, K, M):
         assert hlq.rel_fro_error(y32[m], ref[m]) <= 2 * TOL_F32
     y16 = gemm_f16(X, packed, N, K)                                # default path
     assert hlq.rel_fro_error(y16, ref) <= TOL_F16
-    if M < 16 or G != 128:                               # below the tensor-core threshold: the same kernels
+    if M < 9 or G != 128:                                # below the tensor-core threshold: the same kernels
         assert np.array_equal(y16.view(np.uint16), y32.astype(np.float16).view(np.uint16))
 
 
@@ -78,7 +78,7 @@ def test_prefill_sized_batch_on_a_layer_sized_matrix():
     X = synth.activations(23, "prefill/x", M, K)
     packed = pack_layer(layer)
     ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
-    y16 = gemm_f16(X, packed, N, K)                                  # default path for M >= 16: tensor cores
+    y16 = gemm_f16(X, packed, N, K)                                  # default path for M >= 9: tensor cores
     assert hlq.rel_fro_error(y16, ref) <= TOL_F16
     y32 = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)           # look-up-table kernels
     assert hlq.rel_fro_error(y32, ref) <= TOL_F32

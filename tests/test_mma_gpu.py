@@ -1,4 +1,4 @@
-"""GPU parity of the tensor-core (dequantise-and-contract) path for batches of 16 rows or more.
+"""GPU parity of the tensor-core (dequantise-and-contract) path for batches of 9 rows or more.
 
 Tolerance: the path rebuilds W_hat in fp16 (the BCQ form: z^ rounded once, then one fused multiply-add
 per plane, each rounding at 2^-11 relative), multiplies exactly and accumulates in fp32.  The weight
@@ -22,7 +22,7 @@ from gpu_util import gemm_f16, gemm_f32, pack_layer, x_dev  # noqa: E402
 TOL = 1e-3
 
 # (q, N, K, M): one tile, ragged N / M / K tails, every q, several token tiles, a K split
-CASES = [(2, 512, 1024, 16), (3, 300, 1536, 40), (2, 256, 512, 64), (2, 200, 1024, 100), (3, 1000, 1536, 128), (4, 384, 2560, 300),
+CASES = [(2, 300, 1024, 9), (2, 512, 1024, 16), (3, 300, 1536, 40), (2, 256, 512, 64), (2, 200, 1024, 100), (3, 1000, 1536, 128), (4, 384, 2560, 300),
          (1, 130, 640, 65), (2, 4096, 4096, 128), (3, 512, 4096, 700),
          (2, 4096, 512, 2560)]      # 160 tiles: whole rounds plus a K-split tail stripe
 
