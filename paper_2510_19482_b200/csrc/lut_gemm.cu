@@ -210,8 +210,18 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
     const int bid = blockIdx.x;
-    const int first = bid * a.items_q + min(bid, a.items_r);
-    const int last = first + a.items_q + (bid < a.items_r ? 1 : 0);
+    // CTA b owns a contiguous range of the item list: either an even cut of the whole list, or (aligned partition,
+    // ranges > 0) one of `ranges` row ranges of a single (row batch, half chunk) segment, so that it builds its
+    // tables exactly once.
+    int first, last;
+    if (a.ranges > 0) {
+        const int seg = bid / a.ranges, r = bid - seg * a.ranges;
+        first = seg * a.n_rb + r * a.rb_q + min(r, a.rb_r);
+        last = first + a.rb_q + (r < a.rb_r ? 1 : 0);
+    } else {
+        first = bid * a.items_q + min(bid, a.items_r);
+        last = first + a.items_q + (bid < a.items_r ? 1 : 0);
+    }
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
     const int n_kc2 = 2 * a.n_kc;
@@ -362,6 +372,19 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     b.items_r = (int)(total % grid);
     b.active_warps = kWarps;
     b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1; b.cluster_reduce = 0;
+    // Aligned partition when every (row batch, half chunk) segment can have its own CTAs: a CTA that straddles two
+    // segments builds two table sets, which costs more than the slightly uneven ranges.
+    const long long n_seg = (long long)n_mb * 2 * a.n_kc;
+    if (n_seg <= num_sms && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
+        int R = (int)(num_sms / n_seg);
+        if (R > a.n_rb) R = a.n_rb;
+        if (R >= 1 && n_seg * R * 10 >= (long long)num_sms * 9) {      // only while it still uses >= 90 % of the SMs
+            b.ranges = R;
+            b.rb_q = a.n_rb / R;
+            b.rb_r = a.n_rb % R;
+            grid = n_seg * R;
+        }
+    }
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
