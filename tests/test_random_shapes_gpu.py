@@ -1,0 +1,44 @@
+"""Seeded sweep over odd shapes through every dispatch path (decode, batched look-up, tensor cores) against the
+fp64 oracle: ragged N, K that is not a multiple of 512, M on both sides of each threshold, every q and G."""
+import numpy as np
+import pytest
+
+import paper_2510_19482_b200 as elutq
+import workloads
+from oracle import hlq
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import gemm_f16, gemm_f32, pack_layer  # noqa: E402
+
+
+def _cases():
+    rng = np.random.default_rng(20251019)
+    out = []
+    for i in range(48):
+        q = int(rng.integers(1, 5))
+        G = int(rng.choice([32, 64, 128]))
+        K = G * int(rng.integers(1, 2048 // G + 1))
+        N = int(rng.choice([1, 7, 16, 17, 100, 255, 256, 257, 300, 513, 777]))
+        M = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 10, 15, 16, 17, 31, 33, 64, 127, 128, 129, 200, 257]))
+        out.append((i, q, G, N, K, M))
+    return out
+
+
+@pytest.mark.parametrize("i,q,G,N,K,M", _cases())
+def test_random_shape(i, q, G, N, K, M):
+    layer = workloads.hlq_layer(50 + i, f"rand/{i}", q, G, N, K, signed_scales=(i % 3 == 0))
+    X = synth.activations(50 + i, f"rand/x/{i}", M, K, outliers=(i % 4 == 0))
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    tensor_path = M >= 9 and G == 128
+    y32 = gemm_f32(X, packed, N, K)
+    assert np.all(np.isfinite(y32))
+    assert hlq.rel_fro_error(y32, ref) <= (1e-3 if tensor_path else 5e-6)
+    y16 = gemm_f16(X, packed, N, K)
+    assert hlq.rel_fro_error(y16, ref) <= 1e-3
+    if tensor_path:
+        ylut = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)
+        assert hlq.rel_fro_error(ylut, ref) <= 5e-6
+    assert elutq.elutq_device_status() == 0
