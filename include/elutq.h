@@ -80,6 +80,13 @@ typedef enum elutq_status {
                                       lossy variant: each entry carries a 2^-11 relative rounding (about 3e-4
                                       on Y).  Stays on the look-up kernels at every M; ignored at M = 1          */
 
+#define ELUTQ_FLAG_TABLE_I8 0x200u  /* M >= 2, G = 128: table quantisation of Appendix D, second form - the look-up
+                                      tables hold int8 entries (round to nearest of entry / scale, one scale per
+                                      activation row and 128-column group = largest possible |entry| / 127), 8 rows
+                                      per 8-byte load, integer accumulation inside a group.  Lossy by design: about
+                                      5e-3 relative error on Y, outside the 1e-3 bar of the other paths.  Not
+                                      combinable with ELUTQ_FLAG_TABLE_F16; ignored at M = 1                     */
+
 #define ELUTQ_HEADER_BYTES 128
 
 /* Human-readable name of a status code (static string, never NULL). */

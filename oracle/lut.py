@@ -102,6 +102,40 @@ def table_f16_lut_matmul(X, planes, scales, offsets, G: int, g: int = 8) -> np.n
     return Y
 
 
+def table_i8_lut_matmul(X, planes, scales, offsets, G: int, g: int = 8) -> np.ndarray:
+    """Table quantisation, second form (Appendix D): the table values are mapped to int8.
+
+    The paper fixes no scale; the reading taken here (and by the CUDA variant): one scale per activation
+    row and quantisation group, scale = A / 127 with A the largest magnitude an entry of the group can
+    take (the maximum over the group's slices of sum_i |x_i|), code = round-to-nearest-even(entry / scale)
+    in [-127, 127], looked-up value = code * scale.  Look-ups of a group are summed as integers, then
+    scaled; plane scales and the offset term (from the unquantised group sums) as in lut_matmul.  fp64."""
+    X64 = np.asarray(X, dtype=np.float64)
+    M, K = X64.shape
+    q, N, _ = planes.shape
+    if G % g != 0 or K % G != 0:
+        raise ValueError("need g | G | K")
+    s = np.asarray(scales, dtype=np.float64)
+    z = np.asarray(offsets, dtype=np.float64)
+    idx = plane_indices(planes, g)
+    T = K // g
+    t_ar = np.arange(T)[None, :]
+    Y = np.zeros((M, N), dtype=np.float64)
+    for m in range(M):
+        lut = build_lut(X64[m], g)                                             # [T, 2^g]
+        amax = np.abs(X64[m]).reshape(K // G, G // g, g).sum(axis=2).max(axis=1)   # [groups]
+        sc = amax / 127.0
+        inv = np.where(amax > 0, 127.0 / np.where(amax > 0, amax, 1.0), 0.0)
+        codes = np.rint(lut * np.repeat(inv, G // g)[:, None]).astype(np.int64)     # [T, 2^g]
+        for j in range(q):
+            looked = codes[t_ar, idx[j]]                                        # [N, T] integers
+            acc = looked.reshape(N, K // G, G // g).sum(axis=2)                 # integer sums per group
+            Y[m] += (s[:, :, j] * (acc * sc[None, :])).sum(axis=1)
+        S = lut[:, (1 << g) - 1].reshape(K // G, G // g).sum(axis=1)
+        Y[m] += z @ S
+    return Y
+
+
 def mirror_transform(scales, offsets):
     """(s, z) -> (s^, z^) of Appendix D: s^ = s/2, z^ = z + (1/2) sum_j s_j, in fp64."""
     s = np.asarray(scales, dtype=np.float64)

@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     FLAG_MIRROR,
     FLAG_LUT_ONLY,
     FLAG_TABLE_F16,
+    FLAG_TABLE_I8,
     lib,
     library_path,
     elutq_packed_bytes,

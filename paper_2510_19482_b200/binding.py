@@ -18,6 +18,7 @@ FLAG_CLUSTER_REDUCE = 0x20
 FLAG_MIRROR = 0x40
 FLAG_LUT_ONLY = 0x80
 FLAG_TABLE_F16 = 0x100
+FLAG_TABLE_I8 = 0x200
 
 
 class ElutqError(RuntimeError):

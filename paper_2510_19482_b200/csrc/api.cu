@@ -126,13 +126,14 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     if (!X || !packed || !Y) return ELUTQ_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
     if ((flags & ELUTQ_FLAG_SKIP_OFFSET) && (flags & ELUTQ_FLAG_OFFSET_ONLY)) return ELUTQ_ERR_INVALID_ARG;
-    if (flags & ~0x1ffu) return ELUTQ_ERR_INVALID_ARG;
+    if (flags & ~0x3ffu) return ELUTQ_ERR_INVALID_ARG;
+    if ((flags & ELUTQ_FLAG_TABLE_F16) && (flags & ELUTQ_FLAG_TABLE_I8)) return ELUTQ_ERR_INVALID_ARG;
     if ((flags & ELUTQ_FLAG_PLAIN_G4) && (flags & ELUTQ_FLAG_MIRROR)) return ELUTQ_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(packed, 16) || !aligned(Y, 16)) return ELUTQ_ERR_ALIGN;
     BlobMeta m;
     int st = lookup_blob(packed, N, K, &m);
     if (st != ELUTQ_OK) return st;
-    if ((flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_TABLE_F16)) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
+    if ((flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8)) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
 
     const size_t cb = counters_bytes(M, N), pb = partials_bytes(M, N, K);
     void* counters = workspace;
@@ -162,7 +163,7 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     const int sms = num_sms();
     int ce;
     const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY |
-                                  ELUTQ_FLAG_TABLE_F16;
+                                  ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8;
     if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
     else if (M >= (debug_env("ELUTQ_DEBUG_MMA_MIN_M") > 0 ? debug_env("ELUTQ_DEBUG_MMA_MIN_M") : ELUTQ_TENSOR_MIN_M) && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
     else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);

@@ -20,18 +20,20 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kHalfK = 256;                        // input columns covered by one table set
 
-// TH = true: half-precision tables (table quantisation of Appendix D, first form): an entry holds MB fp16
-// values, so one 8- or 16-byte load serves 4 or 8 activation rows.
-template <int Q, int G, int MB, bool TH = false>
+// TQ selects the table entry format (table quantisation of Appendix D): 0 = fp32 (MB floats per entry);
+// 1 = fp16 (first form: MB halves per entry, one 8- or 16-byte load serves 4 or 8 activation rows);
+// 2 = int8 (second form, lossy: MB = 8 biased bytes per entry, one scale per activation row and 128-column group).
+template <int Q, int G, int MB, int TQ = 0>
 struct BCfg {
     static constexpr int W = G / 8;
     static constexpr int NSG = 128 / G;
     static constexpr int NPW = 2 * NSG * (Q + 1) / 2;          // parameter words per lane (both halves)
     static constexpr int PLANE_BYTES = 1024 * Q;
     static constexpr int TILE_BYTES = PLANE_BYTES + 128 * NPW;
-    static constexpr int ENTRY_BYTES = (TH ? 2 : 4) * MB;      // one table entry: MB floats (or halves)
+    static constexpr int ENTRY_BYTES = (TQ == 0 ? 4 : TQ == 1 ? 2 : 1) * MB;
     static constexpr int TABLE_BYTES = 256 * 32 * ENTRY_BYTES; // 64 KiB (8-byte entries) or 128 KiB (16-byte entries)
-    static constexpr int SMEM_BYTES = TABLE_BYTES + (256 / G) * MB * 4 + 64;
+    // + group sums [256/G][MB] (+ for int8 the row scales [2][MB]) + slack
+    static constexpr int SMEM_BYTES = TABLE_BYTES + (256 / G) * MB * 4 + (TQ == 2 ? 2 * MB * 4 : 0) + 64;
 };
 
 // Tables of half chunk kc2 for rows m0 .. m0+MB-1: lane -> column c (8 activations of every row),
@@ -201,9 +203,105 @@ __device__ __forceinline__ void build_tables_half(uint8_t* smem, int table_bytes
     }
 }
 
-template <int Q, int G, int MB, bool TH>
+// int8 tables for rows m0 .. m0+7 at G = 128 (the half chunk holds two groups of 16 byte-columns): per row and group
+// one scale = (largest possible |entry| of the group, i.e. max over its columns of sum_i |x_i|) / 127; an entry is
+// round-to-nearest(entry / scale) + 128, one byte per row.  Group sums (offset term) stay in fp32.
+__device__ __forceinline__ void build_tables_i8(uint8_t* smem, int table_bytes, const __half* __restrict__ X,
+                                                int M, int K, int m0, int kc2, int tid) {
+    constexpr int MB = 8, W = 16;
+    float* gsum = reinterpret_cast<float*>(smem + table_bytes);   // [2 groups][MB]
+    float* rscale = gsum + 2 * MB;                                // [2 groups][MB]
+    const int lane = tid & 31, warp = tid >> 5;
+    const int hi = warp & 15, lh = warp >> 4;
+    const int k0 = kc2 * kHalfK + lane * 8;
+    uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * MB + lane * MB;
+#pragma unroll 1
+    for (int quad = 0; quad < 2; ++quad) {
+        float2 x[2][8];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            float xa[8], xb[8];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int m = m0 + 4 * quad + 2 * p + r;
+                float* dst = r ? xb : xa;
+                if (m < M && k0 < K) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                        dst[2 * i] = f.x;
+                        dst[2 * i + 1] = f.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
+        }
+        float2 A[2][8], Bv[2], e7[2], inv[2];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            // largest |entry| this column can produce, then the group's maximum over its 16 columns
+            float ax = 0.f, ay = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { ax += fabsf(x[p][i].x); ay += fabsf(x[p][i].y); }
+#pragma unroll
+            for (int off = W / 2; off >= 1; off >>= 1) {
+                ax = fmaxf(ax, __shfl_xor_sync(0xffffffffu, ax, off));
+                ay = fmaxf(ay, __shfl_xor_sync(0xffffffffu, ay, off));
+            }
+            inv[p] = make_float2(ax > 0.f ? 127.f / ax : 0.f, ay > 0.f ? 127.f / ay : 0.f);
+            if (warp == 31 && (lane % W) == 0) {
+                rscale[(lane / W) * MB + 4 * quad + 2 * p] = ax / 127.f;
+                rscale[(lane / W) * MB + 4 * quad + 2 * p + 1] = ay / 127.f;
+            }
+            A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
+            A[p][1] = fadd2(A[p][0], x[p][0]);
+            A[p][2] = fadd2(A[p][0], x[p][1]);
+            A[p][3] = fadd2(A[p][1], x[p][1]);
+            A[p][4] = fadd2(A[p][0], x[p][2]);
+            A[p][5] = fadd2(A[p][1], x[p][2]);
+            A[p][6] = fadd2(A[p][2], x[p][2]);
+            A[p][7] = fadd2(A[p][3], x[p][2]);
+            Bv[p] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const float2 ea = fadd2(A[0][t], Bv[0]), eb = fadd2(A[1][t], Bv[1]);
+            const uint32_t c0 = (uint32_t)(__float2int_rn(ea.x * inv[0].x) + 128), c1 = (uint32_t)(__float2int_rn(ea.y * inv[0].y) + 128);
+            const uint32_t c2 = (uint32_t)(__float2int_rn(eb.x * inv[1].x) + 128), c3 = (uint32_t)(__float2int_rn(eb.y * inv[1].y) + 128);
+            *reinterpret_cast<uint32_t*>(rowp + (size_t)t * 32 * MB + quad * 4) = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+            if (t == 7) { e7[0] = ea; e7[1] = eb; }
+        }
+        if (warp == 31) {   // entry 255: the column's activation sums; reduce over the 16 columns of a group
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                float sx = e7[p].x, sy = e7[p].y;
+#pragma unroll
+                for (int off = W / 2; off >= 1; off >>= 1) {
+                    sx += __shfl_xor_sync(0xffffffffu, sx, off);
+                    sy += __shfl_xor_sync(0xffffffffu, sy, off);
+                }
+                if ((lane % W) == 0) {
+                    gsum[(lane / W) * MB + 4 * quad + 2 * p] = sx;
+                    gsum[(lane / W) * MB + 4 * quad + 2 * p + 1] = sy;
+                }
+            }
+        }
+    }
+}
+
+template <int Q, int G, int MB, int TQ>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a) {
-    using C = BCfg<Q, G, MB, TH>;
+    using C = BCfg<Q, G, MB, TQ>;
+    constexpr bool TH = (TQ == 1);
     extern __shared__ __align__(1024) uint8_t smem[];
     const float* gsum = reinterpret_cast<const float*>(smem + C::TABLE_BYTES);
 
@@ -255,7 +353,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
         const int m0 = mb * MB;
         const int u = kc2 & 1;
         __syncthreads();
-        if (TH) build_tables_half<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
+        if constexpr (TQ == 2) build_tables_i8(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
+        else if constexpr (TQ == 1) build_tables_half<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
         else build_tables_mb<G, MB>(smem, C::TABLE_BYTES, a.X, a.M, a.K, m0, kc2, tid);
         __syncthreads();
 
@@ -293,6 +392,30 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
                     const uint32_t wd[4] = {vec[j].x, vec[j].y, vec[j].z, vec[j].w};
 #pragma unroll
                     for (int v = 0; v < C::NSG; ++v) {
+                        if constexpr (TQ == 2) {
+                            // int8 entries: rows (0,2) / (1,3) / (4,6) / (5,7) accumulate as pairs of 16-bit lanes
+                            // (16 look-ups of at most 255 each cannot carry), then each row is un-biased, converted
+                            // and scaled by (row scale of the group) x (plane scale)
+                            uint32_t ai[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                            for (int ii = 0; ii < C::W; ++ii) {
+                                const uint32_t off = prmt(wd[ii >> 2], colp[ii / 3], 0x7704 + 0x10 * (ii & 3) + (ii % 3));
+                                const uint2 e = *reinterpret_cast<const uint2*>(smem + off);
+                                ai[0] += e.x & 0x00ff00ffu;
+                                ai[1] += (e.x >> 8) & 0x00ff00ffu;
+                                ai[2] += e.y & 0x00ff00ffu;
+                                ai[3] += (e.y >> 8) & 0x00ff00ffu;
+                            }
+                            const float s = prm[v * (Q + 1) + j];
+                            const float* rs = reinterpret_cast<const float*>(smem + C::TABLE_BYTES) + 2 * MB + h * MB;
+#pragma unroll
+                            for (int m = 0; m < MB; ++m) {
+                                const uint32_t word = ai[(m >> 2) * 2 + (m & 1)];
+                                const int code_sum = (int)((m & 2) ? (word >> 16) : (word & 0xffffu)) - C::W * 128;
+                                y[m] = fmaf(s * rs[m], (float)code_sum, y[m]);
+                            }
+                            continue;
+                        }
                         float2 acc[MB / 2];
 #pragma unroll
                         for (int p = 0; p < MB / 2; ++p) acc[p] = make_float2(0.f, 0.f);
@@ -350,14 +473,14 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
     }
 }
 
-template <int Q, int G, int MB, bool TH = false>
+template <int Q, int G, int MB, int TQ = 0>
 int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    using C = BCfg<Q, G, MB, TH>;
+    using C = BCfg<Q, G, MB, TQ>;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(lut_gemm_kernel<Q, G, MB, TH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(lut_gemm_kernel<Q, G, MB, TQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
     }
@@ -396,7 +519,7 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB, TH>, b);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB, TQ>, b);
     count_launch(1);
     if (e != cudaSuccess) return (int)e;
     return launch_finalize(b, 2 * a.n_kc, cfg.numAttrs != 0, stream);
@@ -404,9 +527,13 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
 
 template <int Q, int G>
 int launch_qg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
+    if (a.flags & ELUTQ_FLAG_TABLE_I8) {
+        if constexpr (G == 128) return launch_mb<Q, G, 8, 2>(a, num_sms, stream);
+        else return (int)cudaErrorNotSupported;
+    }
     if (a.flags & ELUTQ_FLAG_TABLE_F16) {
         if constexpr (G == 128)
-            return a.M <= 4 ? launch_mb<Q, G, 4, true>(a, num_sms, stream) : launch_mb<Q, G, 8, true>(a, num_sms, stream);
+            return a.M <= 4 ? launch_mb<Q, G, 4, 1>(a, num_sms, stream) : launch_mb<Q, G, 8, 1>(a, num_sms, stream);
         else
             return (int)cudaErrorNotSupported;
     }

@@ -61,7 +61,8 @@ def test_pointer_validation_happens_before_any_launch():
     assert L.elutq_lut_gemm(16, 16, 16, 0, 16, 512, None) == -1
     assert L.elutq_lut_gemm(8, 16, 16, 1, 16, 512, None) == -3
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x3, 16, 1 << 20, None) == -1   # skip-offset + offset-only
-    assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x200, 16, 1 << 20, None) == -1
+    assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x400, 16, 1 << 20, None) == -1
+    assert L.elutq_lut_gemm_ws(16, 16, 16, 4, 16, 512, 0x300, 16, 1 << 20, None) == -1      # fp16 + int8 tables
     assert L.elutq_lut_gemm_ws(16, 16, 16, 1, 16, 512, 0x50, 16, 1 << 20, None) == -1       # plain g4 + mirror
     assert L.elutq_hlq_fit(None, 2, 128, 16, 512, 10, None, None, None, None, None) == -1
     assert L.elutq_hlq_fit(16, 2, 128, 16, 512, 0, 16, 16, 16, None, None) == -1          # t_max < 1

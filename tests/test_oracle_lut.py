@@ -100,3 +100,41 @@ def test_f16_tables_error_is_one_rounding_per_entry():
     assert np.all(np.abs(got - ref) <= bound)
     assert np.any(got != ref)
     assert hlq.rel_fro_error(got, ref) < 1e-3
+
+
+def test_i8_tables_are_exact_when_entries_sit_on_the_code_grid():
+    """Activations that are multiples of 1/16 with one slice per group summing to 127/16 in magnitude: the scale is
+    exactly 1/16, every table entry is an integer number of scales, so the int8-table procedure is lossless and
+    must reproduce the definition exactly."""
+    rng = np.random.default_rng(10)
+    q, G, N, K, M = 2, 64, 9, 256, 2
+    X = (rng.integers(-12, 13, size=(M, K)) / 16.0)
+    for m in range(M):
+        for gi in range(K // G):
+            X[m, gi * G: gi * G + 8] = [1, -1, 1, 1, -1, 1, 1, 0.9375]        # sum |x| = 127/16, the group's maximum
+    X = X.astype(np.float16)
+    assert np.abs(X.astype(np.float64)).reshape(M, K // 8, 8).sum(axis=2).max() == 127 / 16
+    planes = rng.integers(0, 2, size=(q, N, K)).astype(np.uint8)
+    scales = rng.integers(-4, 5, size=(N, K // G, q)).astype(np.float16)
+    offsets = rng.integers(-3, 4, size=(N, K // G)).astype(np.float16)
+    ref = hlq.matmul(X, planes, scales, offsets, G)
+    assert np.array_equal(lut.table_i8_lut_matmul(X, planes, scales, offsets, G), ref)
+
+
+def test_i8_tables_error_is_half_a_code_per_lookup():
+    """General activations: each looked-up value is off by at most scale / 2, so the deviation from the definition
+    is bounded by sum |s| * (slices per group) * scale / 2; it is far larger than the fp16-table error."""
+    rng = np.random.default_rng(11)
+    q, G, N, K, M = 3, 128, 10, 512, 2
+    planes = rng.integers(0, 2, size=(q, N, K)).astype(np.uint8)
+    scales = np.abs(rng.normal(0, 0.02, size=(N, K // G, q))).astype(np.float16)
+    offsets = rng.normal(0, 0.01, size=(N, K // G)).astype(np.float16)
+    X = rng.normal(0, 1, size=(M, K)).astype(np.float16)
+    ref = hlq.matmul(X, planes, scales, offsets, G)
+    got = lut.table_i8_lut_matmul(X, planes, scales, offsets, G)
+    amax = np.abs(X.astype(np.float64)).reshape(M, K // G, G // 8, 8).sum(axis=3).max(axis=2)   # [M, groups]
+    bound = np.einsum("mg,ngj->mn", amax / 127.0 / 2.0 * (G // 8), np.abs(scales.astype(np.float64)))
+    assert np.all(np.abs(got - ref) <= bound * (1 + 1e-12))
+    e8 = hlq.rel_fro_error(got, ref)
+    e16 = hlq.rel_fro_error(lut.table_f16_lut_matmul(X, planes, scales, offsets, G), ref)
+    assert 1e-3 < e8 < 3e-2 and e8 > 5 * e16
