@@ -474,7 +474,7 @@ def run_cuda(args) -> None:
                 "peak_source": peak_src,
                 "traffic": traffic.get("dram_bytes_per_step") if traffic else None,
                 "traffic_note": traffic.get("note") if traffic else None}
-    tensor_path = all(c.M >= 64 and c.G == 128 for c in calls) and not (args.flags & 0xF0)
+    tensor_path = all(c.M >= 9 and c.G == 128 for c in calls) and not (args.flags & 0x3F0)   # ELUTQ_TENSOR_MIN_M
     if tensor_path:
         # every call of the step is a dense contraction on the tensor cores: report FLOP/s against the measured
         # GEMM peak (the sustained figure, since the kernels are timed inside a long step)

@@ -1,4 +1,4 @@
-// Prefill-sized batches (M >= 64): dequantise-and-contract on the 5th-generation tensor cores.
+// Batches of ELUTQ_TENSOR_MIN_M rows or more at G = 128: dequantise-and-contract on the 5th-generation tensor cores.
 //
 // For large M the look-up path is bound by the shared-memory look-up rate (it does M look-ups per
 // weight byte), while Y = X W_hat^T is then a genuine dense contraction.  This kernel rebuilds each
