@@ -1,15 +1,18 @@
-// M > 1: small-batch / prefill LUT GEMM over the same packed layout.
+// 2 <= M < ELUTQ_TENSOR_MIN_M (or any M > 1 on request): batched look-up GEMM over the same packed layout.
 //
-// MB activation rows (2 or 4) are processed per pass: a table entry holds the partial sums of all MB
-// rows for one (byte value, column), so one weight byte costs one byte-permute, one 8- or 16-byte
-// shared-memory load and MB/2 packed fp32x2 adds.  Tables of one pass cover half a tile (256 input
-// columns = super-groups 2u and 2u+1 of a chunk): 256 entries x 32 columns x MB floats.
+// MB activation rows are processed per pass: a table entry holds the partial sums of all MB rows for one
+// (byte value, column), so one weight byte costs one byte-permute, one shared-memory load and the adds of MB
+// rows.  fp32 tables: MB = 2 or 4 (8- or 16-byte entries, packed fp32x2 adds).  Quantised tables of Appendix D
+// as labelled variants: fp16 entries (MB = 4 or 8, converted and added in fp32) and int8 entries (MB = 8, one
+// scale per row and group, integer adds in 16-bit lanes).  Tables of one pass cover half a tile (256 input
+// columns = super-groups 2u and 2u+1 of a chunk): 256 entries x 32 columns.
 //
-// Work list: (row batch mb, half chunk kc2 = 2*kc + u, row block rb), flattened in that order and cut
-// into equal contiguous ranges, one per CTA (one 1024-thread CTA per SM); tables are rebuilt when a
-// range crosses an (mb, kc2) boundary.  Partial sums go to partials[kc2][m][n]; the finalize kernel adds
-// the 2*n_kc half chunks in ascending order.  The look-up rate of shared memory (one 4-byte entry per
-// lane per cycle per SM), not HBM, bounds this path: time grows with M.
+// Work list: (row batch mb, half chunk kc2 = 2*kc + u, row block rb), flattened in that order.  A CTA (one
+// 1024-thread CTA per SM) owns a row range of one (mb, kc2) segment and builds its tables once (aligned
+// partition), or, when that would idle more than a tenth of the SMs, an equal contiguous cut of the whole list
+// (tables are rebuilt when the cut crosses a segment boundary).  Partial sums go to partials[kc2][m][n]; the
+// finalize kernel adds the 2*n_kc half chunks in ascending order.  With fp32 tables the shared-memory look-up
+// rate (one 4-byte entry per lane per cycle per SM), not HBM, bounds this path: time grows with M.
 #include "common.cuh"
 
 namespace elutq {
