@@ -190,7 +190,10 @@ int elutq_lut_gemm_ws(const void* X, const void* packed, void* Y, int M, int N, 
  * device, the product runs, and Y (fp16 [M][N]) is copied back to Y_host, all on
  * `stream` (use pinned host memory for the copies to be asynchronous).  `packed`
  * stays a device pointer.  Staging buffers are library-owned like the scratch of
- * elutq_lut_gemm.  The call returns without synchronising.
+ * elutq_lut_gemm.  The call returns without synchronising.  When both host buffers are pinned and
+ * addressable by the device and together at most 1 MiB (decode, small batches), X is pulled across the
+ * bus by a small kernel and Y is stored straight into host memory by the epilogue (no copy-engine
+ * operations, which cost several microseconds each); otherwise two cudaMemcpyAsync are used.
  */
 int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
                         int M, int N, int K, void* stream);
