@@ -293,6 +293,8 @@ def run_cuda(args) -> None:
     copies = max(1, min(8, -(-3 * l2_bytes // max(working_set, 1))))
     if copies * working_set > (16 << 30):
         copies = 1
+    if os.environ.get("ELUTQ_BENCH_COPIES"):          # experiments: e.g. 1 keeps a small working set L2-resident
+        copies = max(1, int(os.environ["ELUTQ_BENCH_COPIES"]))
     layer_sets = [layers]
     for _ in range(1, copies):
         dup = []

@@ -179,7 +179,10 @@ __device__ __forceinline__ float sum_chunks(const float* p, size_t stride, int n
     return sum;
 }
 
-template <int Q, int G, int MODE>
+// FAST = the common call shape fixed at compile time (both terms, aligned partition with one chunk per CTA, K split
+// reduced by the finalize kernel): the flag tests, the segment arithmetic and the other reduction forms drop out
+// of the item loop.
+template <int Q, int G, int MODE, bool FAST = false>
 __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a) {
     using C = Cfg<Q, G>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -208,8 +211,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         first = bid * a.items_q + min(bid, a.items_r);
         last = first + a.items_q + (bid < a.items_r ? 1 : 0);
     }
-    const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
-    const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
+    const bool use_planes = FAST || !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
+    const bool use_offset = FAST || !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
     // Byte offset (< 128) of the lane's column inside a 256-byte table row, per step, four steps
     // per register: the byte-permute below picks byte (i & 3) of colp[i >> 2] as address byte 0,
@@ -352,10 +355,10 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
             y += __shfl_xor_sync(0xffffffffu, y, 16);
 
             const int row = (it - kc * a.n_rb) * kTileRows + l;
-            if (a.n_kc == 1) {
+            if (!FAST && a.n_kc == 1) {
                 if (h == 0 && row < a.N) store_out(a, (size_t)row, y);
             } else if (h == 0) {
-                if (a.cluster_reduce) cpart[row - range_rb0 * kTileRows] = y;
+                if (!FAST && a.cluster_reduce) cpart[row - range_rb0 * kTileRows] = y;
                 else a.partials[(size_t)kc * n_pad + row] = y;
             }
         };
@@ -363,8 +366,8 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         while (it < seg_end) {
             // next item of this warp: `stride` positions further in the concatenated segments
             int nit = it + stride, nend = it_end;
-            while (nit >= nend && nend < last) { nit += jump; nend += a.n_rb; }
-            const bool has_next = nit < nend && !(a.flags & 0x80000000u);
+            if (!FAST) while (nit >= nend && nend < last) { nit += jump; nend += a.n_rb; }
+            const bool has_next = nit < nend && (FAST || !(a.flags & 0x80000000u));
             nvp = a.tiles + (size_t)nit * C::TILE_BYTES + lane * 16;
             npp = nvp + (C::PLANE_BYTES - lane * 12);
             if (has_next) do_item(IntC<1>{});
@@ -376,7 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
         seg = (a.ranges > 0) ? seg + a.n_rb : seg_end;
     }
 
-    if (a.cluster_reduce && !(a.flags & 0x40000000u)) {
+    if (!FAST && a.cluster_reduce && !(a.flags & 0x40000000u)) {
         // K-split reduction inside the cluster: every CTA holds the partial sums of its chunk for the
         // cluster's row range in shared memory; after the cluster barrier CTA c adds, for its share of the
         // rows, the n_kc partials in ascending chunk order (bit-reproducible) straight from its peers'
@@ -394,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
             if (row < a.N) store_out(a, (size_t)row, sum);
         }
         cluster_barrier();          // nobody leaves while a peer may still read its shared memory
-    } else if (a.fused_reduce && a.n_kc > 1) {
+    } else if (!FAST && a.fused_reduce && a.n_kc > 1) {
         // In-kernel K-split reduction: each CTA publishes its partials and takes one ticket for its row
         // range; the CTA that draws the last ticket of the range adds the chunks in ascending order
         // (bit-reproducible) and writes Y.  The counter wraps to zero, ready for the next call.
@@ -626,7 +629,24 @@ int launch_one(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     }
     if (debug_env("ELUTQ_DEBUG_NOLOAD") > 0) b.flags |= 0x80000000u;
     if (debug_env("ELUTQ_DEBUG_SKIP_CLUSTER_REDUCE") > 0) b.flags |= 0x40000000u;   // timing experiment only   // timing experiment: skip reloads (results invalid)
-    cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, MODE>, b);
+    const bool fast = MODE == kModeFused && !use_cluster && b.ranges > 0 && b.cpc == 1 && a.n_kc > 1 && !b.fused_reduce &&
+                      !(b.flags & (ELUTQ_FLAG_SKIP_OFFSET | ELUTQ_FLAG_OFFSET_ONLY | 0xC0000000u)) && debug_env("ELUTQ_DEBUG_NO_FAST") == 0;
+    cudaError_t e;
+    if constexpr (MODE == kModeFused) {
+        if (fast) {
+            static bool configured_fast[64] = {};
+            if (dev >= 0 && dev < 64 && !configured_fast[dev]) {
+                e = cudaFuncSetAttribute(lut_gemv_kernel<Q, G, MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+                if (e != cudaSuccess) return (int)e;
+                configured_fast[dev] = true;
+            }
+            e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, MODE, true>, b);
+        } else {
+            e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, MODE, false>, b);
+        }
+    } else {
+        e = cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, G, MODE, false>, b);
+    }
     count_launch(1);
     if (e != cudaSuccess || a.n_kc == 1 || b.fused_reduce || b.cluster_reduce) return (int)e;
     if (debug_env("ELUTQ_DEBUG_SKIP_FINALIZE") > 0) return (int)e;   // timing experiment only (Y is not written)
