@@ -150,9 +150,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_d = *tmem_slot;
 
-    grid_launch_dependents();
-    grid_dependency_wait();
-
     // instruction descriptor: D = fp32, A = B = fp16, both K-major, M = 128 tokens, N = NW weight rows
     constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NW >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
     const uint32_t x_addr = smem_u32(sX), w_addr = smem_u32(sW), bar_addr = smem_u32(mbar);
@@ -214,6 +211,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             static_for<0, NPW>([&](auto i) { pw[i] = ldg_stream_u32<0>(tile + PLANE_BYTES + (i * 32 + pl) * 4); });
         }
     };
+
+    // The packed weights do not depend on the previous kernel in the stream (X, Y and the partial buffer do):
+    // the first step's vectors are requested before the dependency wait.
+    if (step0 < step1) load_weights(step0);
+    grid_launch_dependents();
+    grid_dependency_wait();
 
     // The packed layout rotates a lane's 16 plane bytes (byte i covers 16-byte column (l + i) mod 16 of the
     // super-group, which keeps the look-up kernels free of bank conflicts).  Here the halves of the weight tile
@@ -355,10 +358,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                          :: "r"(bar_addr + 8u * wt) : "memory");
         };
-        if (step0 < step1) {
-            copy_x(step0, 0);
-            load_weights(step0);
-        }
+        if (step0 < step1) copy_x(step0, 0);
         asm volatile("cp.async.commit_group;" ::: "memory");
         for (int step = step0; step < step1; ++step) {
             const int i = step - step0, wt = i & 1;
@@ -379,10 +379,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) hlq_mma_kernel(const GemmArgs 
         if (n >= 2) wait_mma((n - 2) & 1, (uint32_t)((((n - 2) >> 1)) & 1));
         if (n >= 1) wait_mma((n - 1) & 1, (uint32_t)((((n - 1) >> 1)) & 1));
     } else {
-        if (step0 < step1) {
-            copy_x(step0, 0);
-            load_weights(step0);
-        }
+        if (step0 < step1) copy_x(step0, 0);
         asm volatile("cp.async.commit_group;" ::: "memory");
 
         // Steady state: the tensor core works on one half of the weight tile while the threads dequantise the other.
