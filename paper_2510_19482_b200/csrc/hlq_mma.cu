@@ -106,30 +106,40 @@ __device__ __forceinline__ void store_row32(const GemmArgs& a, int m, int n0, co
 // NW = weight rows per CTA (UMMA N: 128 or 256); TT = token tiles of 128 per CTA (1 or 2).
 // WS (TT = 2 only) = warp-specialised form: a ninth warp issues the MMAs, the eight producer warps hand each finished
 // half over through an mbarrier (one arrival per warp) instead of a CTA-wide barrier.
-template <int Q, int NW, int TT, bool WS = false>
+//
+// CG = 2 (with WS): a pair of CTAs (thread-block cluster of two along the token dimension, one SM pair) works on one
+// weight tile with `tcgen05.mma.cta_group::2`, UMMA M = 256: each CTA holds its own 2 x 128 tokens (A operand rows and
+// accumulator lanes) and dequantises only its half of the tile's weight rows (the tensor core reads the two halves of
+// B from the two CTAs' shared memory), so the dequantisation per MMA is halved.  The issuer warp of the leader CTA
+// (cluster rank 0) waits for the arrivals of all 16 producer warps (the peer's arrive through the cluster window) and
+// commits each half's MMAs to the "done" barriers of both CTAs.
+template <int Q, int NW, int TT, bool WS = false, int CG = 1>
 __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel(const GemmArgs a, const int splits, const int n_tile0) {
     static_assert(!WS || TT == 2, "the warp-specialised form exists for two token tiles only");
+    static_assert(CG == 1 || (WS && CG == 2), "the CTA-pair form builds on the warp-specialised one");
+    constexpr int NWL = NW / CG;                         // weight rows dequantised by this CTA
     constexpr int NPW = Q + 1;                           // parameter words per lane at G = 128
     constexpr int PLANE_BYTES = 1024 * Q;
     constexpr int TILE_BYTES = PLANE_BYTES + 128 * (Q + 1);
-    constexpr int PAIRS = NW / 32;                       // item pairs per step: 8 or 4
+    constexpr int PAIRS = NWL / 32;                      // item pairs per step: 8 or 4
     constexpr int WPP = (kMmaThreads / 32) / PAIRS;      // warps sharing one item pair: 1 or 2
     constexpr int NB = 8 / WPP;                          // plane bytes per lane and half step
-    constexpr int W_HALF_BYTES = NW * 64 * 2;            // one half (64 k) of the weight tile
+    constexpr int W_HALF_BYTES = NWL * 64 * 2;           // one half (64 k) of this CTA's part of the weight tile
     constexpr int X_STAGE_BYTES = TT * kXTileBytes;
-    constexpr int W_BYTES = NW * kStepK * 2;
+    constexpr int W_BYTES = NWL * kStepK * 2;
     constexpr int XS = (TT == 1) ? 3 : 2;                // activation stages
-    constexpr int WB = (TT == 1) ? 2 : 1;                // whole weight tiles (each of two halves)
+    constexpr int WB = (TT == 1 || CG == 2) ? 2 : 1;     // whole weight tiles (each of two halves); the pair form uses them as a ring of four halves
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sX = smem;                                  // A operand stages
     uint8_t* sW = smem + XS * X_STAGE_BYTES;             // B operand
     uint64_t* mbar = reinterpret_cast<uint64_t*>(sW + WB * W_BYTES);        // [2]: one per weight-tile half (TT = 2)
                                                                             //      or per weight tile (TT = 1)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 4);            // mbar[2], mbar[3]: "half is ready" (WS)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 8);            // WS: mbar[2], mbar[3] = "half is ready"; pair form: [0..3] done, [4..7] ready
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int l = lane & 15;
-    const int n_tile = n_tile0 + blockIdx.x, m_tile = blockIdx.y, split = blockIdx.z;
+    // CTA pairs are neighbours in x, so the pair form puts the token tiles there
+    const int n_tile = n_tile0 + (CG == 2 ? blockIdx.y : blockIdx.x), m_tile = (CG == 2 ? blockIdx.x : blockIdx.y), split = blockIdx.z;
     const int m0 = m_tile * (TT * kTileM);
     const int n_steps = 4 * a.n_kc;                                   // super-groups
     const int step0 = (int)((long long)n_steps * split / splits);
@@ -138,25 +148,41 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
     // ---- set-up: tensor memory, completion barriers ---------------------------------------------
+    uint32_t cta_rank = 0;                               // rank in the CTA pair (0 = leader)
+    if constexpr (CG == 2) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)(TT * NW)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (CG == 2) {     // the same warp of both CTAs of the pair allocates (same columns in both)
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)(TT * NW)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)(TT * NW)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar)) : "memory");
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar + 1)) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;" :: "r"(smem_u32(mbar + 2)) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;" :: "r"(smem_u32(mbar + 3)) : "memory");
+        if constexpr (CG == 2) {
+#pragma unroll
+            for (int i = 2; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(mbar + i)) : "memory");
+#pragma unroll
+            for (int i = 4; i < 8; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 16;" :: "r"(smem_u32(mbar + i)) : "memory");
+        } else {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;" :: "r"(smem_u32(mbar + 2)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;" :: "r"(smem_u32(mbar + 3)) : "memory");
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if constexpr (CG == 2) cluster_barrier();            // the peer's barriers are initialised before anyone arrives on them
+    else __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_d = *tmem_slot;
 
     // instruction descriptor: D = fp32, A = B = fp16, both K-major, M = 128 tokens, N = NW weight rows
-    constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NW >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(NW >> 3) << 17) | ((uint32_t)((CG * kTileM) >> 4) << 24);
     const uint32_t x_addr = smem_u32(sX), w_addr = smem_u32(sW), bar_addr = smem_u32(mbar);
 
     // Asynchronous copy of the activation tile(s) of one step into a stage.  Thread (token r = tid / 8 + RPP p,
@@ -204,7 +230,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     const int pair = warp % PAIRS;                        // item pair of this warp
     const int bsel = warp / PAIRS;                        // which NB bytes of the 16 (only when two warps share a pair)
     const int item = 2 * pair + (lane >> 4);
-    const int rb = n_tile * (NW / kTileRows) + item;
+    const int rb = n_tile * (NW / kTileRows) + (int)cta_rank * (NWL / kTileRows) + item;
     uint4 vec[Q];
     uint32_t pw[NPW];
     auto load_weights = [&](int step) {
@@ -251,6 +277,29 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         }
     };
 
+    // The issuer's wait for the producers' arrivals; in a CTA pair the peer's arrivals (and what they release) come
+    // through the cluster, so the wait acquires at cluster scope.
+    auto wait_ready = [&](int which, uint32_t parity) {
+        if (!ok) return;
+        bool done = false;
+        if constexpr (CG == 2) {
+            for (uint32_t i = 0; i < kWaitLimit && !done; ++i) {
+                uint32_t r;
+                asm volatile("{\n\t.reg .pred p;\n\t"
+                             "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                             "selp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(r) : "r"(bar_addr + 8u * which), "r"(parity) : "memory");
+                done = r != 0;
+            }
+        } else {
+            done = mbar_wait(bar_addr + 8u * which, parity);
+        }
+        if (!done) {
+            ok = false;
+            if (a.counters != nullptr) atomicExch(a.counters, 0x7C05u);
+        }
+    };
+
     // Parameters of the step's super-group for this lane's row, decoded once per step: halves
     // [u*(Q+1) .. u*(Q+1)+Q] of the parameter words = s_0..s_{Q-1}, z.
     uint32_t sneg[Q];                                              // (-s_j/2, -s_j/2) as packed fp16
@@ -282,8 +331,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     };
 
     // Dequantise half hb (64 k) of this lane's row into half hb of weight tile wt (BCQ form, in registers).
-    auto dequant_half = [&](int hb, int wt) {
-        uint8_t* buf = sW + wt * W_BYTES + hb * W_HALF_BYTES;
+    auto dequant_half_to = [&](int hb, uint8_t* buf) {
         const uint32_t row_off = (uint32_t)((2 * item + (l >> 3)) * 8) * 128u + (uint32_t)(l & 7) * 16u;
         if (rb < a.n_rb && (use_planes | use_offset)) {
 #pragma unroll
@@ -317,9 +365,11 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         }
     };
 
+    auto dequant_half = [&](int hb, int wt) { dequant_half_to(hb, sW + wt * W_BYTES + hb * W_HALF_BYTES); };
+
     // MMAs of one half step (64 k = 4 slices per token tile), issued by one thread; completion arrives on barrier hb.
     auto issue_mma = [&](int step, int stage, int hb) {
-        if (tid != (WS ? kMmaThreads : 0)) return;
+        if (tid != (WS ? kMmaThreads : 0) || cta_rank != 0) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int tt = 0; tt < TT; ++tt) {
@@ -328,14 +378,26 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + tt * kXTileBytes + hb * (kTileM * 128) + kk * 32);
                 const uint64_t db = desc_noswizzle(w_addr + hb * W_HALF_BYTES + kk * 256);
                 const uint32_t accumulate = (step != step0 || hb != 0 || kk != 0) ? 1u : 0u;
-                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-                             :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
-                             : "memory");
+                if constexpr (CG == 2) {
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                                 : "memory");
+                } else {
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                                 : "memory");
+                }
             }
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                     :: "r"(bar_addr + 8u * hb) : "memory");
+        if constexpr (CG == 2) {     // completion arrives on the same barrier of both CTAs of the pair
+            asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                         :: "r"(bar_addr + 8u * hb), "h"((unsigned short)3) : "memory");
+        } else {
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                         :: "r"(bar_addr + 8u * hb) : "memory");
+        }
     };
     auto publish = [&]() {     // generic-proxy writes of this thread -> visible to the tensor core, then CTA barrier
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -387,12 +449,98 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         // Producer warps: dequantise a half, make it (and the activation stage) visible to the tensor core, arrive on the
         // half's "ready" barrier; before overwriting a half they wait for the MMAs that read it (the "done" barriers).
         // Issuer warp: wait for "ready", issue the half's MMAs, commit them to "done".
-        auto arrive_ready = [&](int hb) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0)
-                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar_addr + 8u * (2 + hb)) : "memory");
+        auto arrive_ready = [&](int bar) {
+            if constexpr (CG == 2) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {     // the leader's barrier, through the cluster window
+                    uint32_t remote;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar_addr + 8u * bar), "r"(0u));
+                    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(remote) : "memory");
+                }
+            } else {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar_addr + 8u * bar) : "memory");
+            }
         };
+        if constexpr (CG == 2) {
+            // CTA pair: half steps i = 0, 1, ... run through rings of four slots (activation half tiles of 2 x 128
+            // tokens x 64 k, and this CTA's 128 weight rows x 64 k); slot i mod 4 has a "ready" barrier (16 producer warps
+            // of the pair, on the leader) and a "done" barrier (the half's MMAs, committed to both CTAs).  The producers run
+            // up to two halves ahead of the MMAs' completion, which hides the hand-over latency through the cluster.
+            constexpr int XH_BYTES = TT * kTileM * 128;          // activation slot
+            constexpr int WH_BYTES = W_HALF_BYTES;               // weight slot
+            const int n_half = 2 * (step1 - step0);
+            auto copy_x_half = [&](int step, int kb, int slot) {
+                const int j = tid & 7, r0 = tid >> 3;
+                const uint32_t dst0 = x_addr + (uint32_t)slot * XH_BYTES + (uint32_t)r0 * 128u + (uint32_t)((j ^ (r0 & 7)) * 16);
+                const int k = step * kStepK + kb * 64;
+                const uint32_t live = (k < a.K) ? x_live : 0u;
+                const int koff = (k < a.K) ? k : 0;
+#pragma unroll
+                for (int tt = 0; tt < TT; ++tt) {
+#pragma unroll
+                    for (int p = 0; p < NPASS; ++p) {
+                        const uint32_t dst = dst0 + (uint32_t)(tt * (kTileM * 128) + p * RPP * 128);
+                        const uint32_t nbytes = ((live >> (tt * NPASS + p)) & 1u) ? 16u : 0u;
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                                     :: "r"(dst), "l"(x_src[tt * NPASS + p] + koff), "r"(nbytes) : "memory");
+                    }
+                }
+            };
+            if (warp < kMmaThreads / 32) {
+                if (n_half > 0) copy_x_half(step0, 0, 0);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                if (n_half > 1) copy_x_half(step0, 1, 1);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                // one half step; hb is a compile-time constant so that the plane words are picked statically
+                auto half_iter = [&](int i, auto hb_c) {
+                    constexpr int hb = decltype(hb_c)::value;
+                    const int step = step0 + (i >> 1), slot = i & 3;
+                    if (hb == 0) {
+                        unrotate();
+                        decode_params(step);
+                    }
+                    // the slot's previous half (i - 4) was waited for two iterations ago
+                    dequant_half_to(hb, sW + slot * WH_BYTES);
+                    if (hb == 1 && step + 1 < step1) load_weights(step + 1);
+                    asm volatile("cp.async.wait_group 1;" ::: "memory");          // the activations of half i have landed
+                    arrive_ready(4 + slot);
+                    if (i >= 2) wait_mma((i - 2) & 3, (uint32_t)(((i - 2) >> 2) & 1));    // slot of half i + 2 is free
+                    if (i + 2 < n_half) copy_x_half(step0 + ((i + 2) >> 1), hb, (i + 2) & 3);
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                };
+                for (int i = 0; i < n_half; i += 2) {
+                    half_iter(i, IntC<0>{});
+                    half_iter(i + 1, IntC<1>{});
+                }
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                if (n_half > 0) wait_mma((n_half - 1) & 3, (uint32_t)(((n_half - 1) >> 2) & 1));   // commits complete in order
+            } else if (cta_rank == 0 && lane == 0) {
+                for (int i = 0; i < n_half; ++i) {
+                    const int slot = i & 3;
+                    wait_ready(4 + slot, (uint32_t)((i >> 2) & 1));
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                    for (int tt = 0; tt < TT; ++tt) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t da = desc_swizzle128(x_addr + slot * XH_BYTES + tt * (kTileM * 128) + kk * 32);
+                            const uint64_t db = desc_noswizzle(w_addr + slot * WH_BYTES + kk * 256);
+                            const uint32_t accumulate = (i != 0 || kk != 0) ? 1u : 0u;
+                            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+                                         :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                                         : "memory");
+                        }
+                    }
+                    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                                 :: "r"(bar_addr + 8u * slot), "h"((unsigned short)3) : "memory");
+                }
+            }
+        } else {
         uint32_t phase = 0;                                   // every barrier completes once per step
         if (warp < kMmaThreads / 32) {
             if (step0 < step1) copy_x(step0, 0);
@@ -404,13 +552,13 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 decode_params(step);
                 dequant_half(0, 0);
                 asm volatile("cp.async.wait_group 0;" ::: "memory");
-                arrive_ready(0);
+                arrive_ready(2);
                 if (step > step0) wait_mma(1, phase ^ 1u);
                 if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 dequant_half(1, 0);
                 if (step + 1 < step1) load_weights(step + 1);
-                arrive_ready(1);
+                arrive_ready(3);
                 phase ^= 1u;
             }
             asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -418,15 +566,16 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 wait_mma(0, phase ^ 1u);
                 wait_mma(1, phase ^ 1u);
             }
-        } else {
+        } else if (cta_rank == 0) {
             for (int step = step0; step < step1; ++step) {
                 const int stage = (step - step0) & 1;
-                wait_mma(2, phase);
+                wait_ready(2, phase);
                 issue_mma(step, stage, 0);
-                wait_mma(3, phase);
+                wait_ready(3, phase);
                 issue_mma(step, stage, 1);
                 phase ^= 1u;
             }
+        }
         }
     } else {
         if (step0 < step1) copy_x(step0, 0);
@@ -490,19 +639,25 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == 0)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"((uint32_t)(TT * NW)) : "memory");
+    if constexpr (CG == 2) {
+        cluster_barrier();           // nobody frees tensor memory or leaves while the pair may still use it
+        if (warp == 0)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"((uint32_t)(TT * NW)) : "memory");
+    } else {
+        __syncthreads();
+        if (warp == 0)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_d), "r"((uint32_t)(TT * NW)) : "memory");
+    }
 }
 
-template <int Q, int NW, int TT, bool WS = false>
+template <int Q, int NW, int TT, bool WS = false, int CG = 1>
 int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
-    constexpr int kSmem = (TT == 1 ? 3 : 2) * TT * kXTileBytes + (TT == 1 ? 2 : 1) * NW * kStepK * 2 + 64;
+    constexpr int kSmem = (TT == 1 ? 3 : 2) * TT * kXTileBytes + (TT == 1 ? 2 : 1) * NW * kStepK * 2 + 128;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(hlq_mma_kernel<Q, NW, TT, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        cudaError_t e = cudaFuncSetAttribute(hlq_mma_kernel<Q, NW, TT, WS, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return (int)e;
         configured[dev] = true;
     }
@@ -513,16 +668,24 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
 
     auto launch = [&](int n_tile0, int n_count, int splits) -> cudaError_t {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)n_count, (unsigned)m_tiles, (unsigned)splits);
+        cfg.gridDim = CG == 2 ? dim3((unsigned)m_tiles, (unsigned)n_count, (unsigned)splits)
+                              : dim3((unsigned)n_count, (unsigned)m_tiles, (unsigned)splits);
         cfg.blockDim = dim3(kMmaThreads + (WS ? 32 : 0));
         cfg.dynamicSmemBytes = kSmem;
         cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = pdl ? 1 : 0;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT, WS>, a, splits, n_tile0);
+        if (CG == 2) {               // CTA pairs along the token dimension (the caller made sure m_tiles is even)
+            attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+            attr[cfg.numAttrs].val.clusterDim.x = 2;
+            attr[cfg.numAttrs].val.clusterDim.y = 1;
+            attr[cfg.numAttrs].val.clusterDim.z = 1;
+            cfg.numAttrs += 1;
+        }
+        cudaError_t e = cudaLaunchKernelEx(&cfg, hlq_mma_kernel<Q, NW, TT, WS, CG>, a, splits, n_tile0);
         count_launch(1);
         return e;
     };
@@ -571,6 +734,9 @@ int launch_mma_q(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     if (debug_env("ELUTQ_DEBUG_MMA_NW") == 128) narrow = true;
     if (debug_env("ELUTQ_DEBUG_MMA_NW") == 256) narrow = false;
     // measured: the warp-specialised form is 3-5 % faster (no CTA-wide barrier in the step, the issuing thread dequantises nothing)
+    // measured: a CTA pair per weight tile (each CTA dequantises half of it) is 8-22 % faster again; it needs an even
+    // number of 256-token tiles
+    if (two && !narrow && m_tiles % 2 == 0 && debug_env("ELUTQ_DEBUG_MMA_NO_PAIR") == 0) return launch_mma_cfg<Q, 256, 2, true, 2>(a, num_sms, stream);
     if (two && !narrow && debug_env("ELUTQ_DEBUG_MMA_NO_WS") == 0) return launch_mma_cfg<Q, 256, 2, true>(a, num_sms, stream);
     if (two) return narrow ? launch_mma_cfg<Q, 128, 2>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 2>(a, num_sms, stream);
     return narrow ? launch_mma_cfg<Q, 128, 1>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 1>(a, num_sms, stream);
