@@ -31,6 +31,13 @@
 //              stores) or, with a K split, to the fp32 partial buffer that the shared finalize kernel
 //              reduces in ascending order.
 //
+//   schedules  M <= 128: one token tile, whole weight tile double-buffered, one CTA barrier per step.  M > 128: two token
+//              tiles per CTA and a ninth warp that issues the MMAs; the eight producer warps hand each dequantised
+//              half over through an mbarrier (one arrival per warp), no CTA-wide barrier in the step.  With an even
+//              number of 256-token tiles the CTAs run as pairs (cluster of two, `cta_group::2`, UMMA M = 256): both
+//              CTAs of a pair work on the same weight tile with their own tokens, each dequantises half of its rows,
+//              and the half steps run through rings of four slots (see the kernel).
+//
 // Every wait is bounded: a thread whose MMA-completion barrier does not flip within the limit raises the
 // status word and stops waiting; it still joins every CTA barrier, and the CTA releases its tensor memory.
 #include "common.cuh"
@@ -451,6 +458,10 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         // Issuer warp: wait for "ready", issue the half's MMAs, commit them to "done".
         auto arrive_ready = [&](int bar) {
             if constexpr (CG == 2) {
+                // Each lane makes its own shared-memory writes visible to the tensor core, the warp converges, lane 0
+                // arrives (release) on the leader's barrier.  The data stay in this CTA's shared memory, where the
+                // tensor core reads them; only the arrival crosses to the peer.  (A cluster-scope release here was
+                // measured 30 % slower for the whole kernel.)
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {     // the leader's barrier, through the cluster window

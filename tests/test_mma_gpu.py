@@ -68,11 +68,16 @@ def test_tensor_core_path_terms_and_accumulate():
     assert elutq.elutq_device_status() == 0
 
 
-def test_tensor_core_path_is_bit_reproducible():
-    q, G, N, K, M = 3, 128, 512, 2048, 128
-    layer = workloads.hlq_layer(32, "mma/repro", q, G, N, K)
-    X = synth.activations(32, "mma/repro/x", M, K)
+@pytest.mark.parametrize("q,N,K,M", [(3, 512, 2048, 128), (2, 4096, 2048, 512), (4, 8192, 1024, 1000)])
+def test_tensor_core_path_is_bit_reproducible(q, N, K, M):
+    """One token tile, and the shapes that run as CTA pairs (hand-over through barriers across two SMs): repeated
+    calls give identical bits, so no half of a weight or activation tile is read before it is complete."""
+    G = 128
+    layer = workloads.hlq_layer(32, f"mma/repro/{q}/{N}", q, G, N, K)
+    X = synth.activations(32, f"mma/repro/x/{M}/{K}", M, K)
     packed = pack_layer(layer)
     a = gemm_f16(X, packed, N, K)
-    b = gemm_f16(X, packed, N, K)
-    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    for _ in range(5):
+        b = gemm_f16(X, packed, N, K)
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    assert elutq.elutq_device_status() == 0
