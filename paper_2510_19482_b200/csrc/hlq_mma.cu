@@ -552,41 +552,41 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 }
             }
         } else {
-        uint32_t phase = 0;                                   // every barrier completes once per step
-        if (warp < kMmaThreads / 32) {
-            if (step0 < step1) copy_x(step0, 0);
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            for (int step = step0; step < step1; ++step) {
-                const int stage = (step - step0) & 1;
-                if (step > step0) wait_mma(0, phase ^ 1u);
-                unrotate();
-                decode_params(step);
-                dequant_half(0, 0);
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                arrive_ready(2);
-                if (step > step0) wait_mma(1, phase ^ 1u);
-                if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
+            uint32_t phase = 0;                                   // every barrier completes once per step
+            if (warp < kMmaThreads / 32) {
+                if (step0 < step1) copy_x(step0, 0);
                 asm volatile("cp.async.commit_group;" ::: "memory");
-                dequant_half(1, 0);
-                if (step + 1 < step1) load_weights(step + 1);
-                arrive_ready(3);
-                phase ^= 1u;
+                for (int step = step0; step < step1; ++step) {
+                    const int stage = (step - step0) & 1;
+                    if (step > step0) wait_mma(0, phase ^ 1u);
+                    unrotate();
+                    decode_params(step);
+                    dequant_half(0, 0);
+                    asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    arrive_ready(2);
+                    if (step > step0) wait_mma(1, phase ^ 1u);
+                    if (step + 1 < step1) copy_x(step + 1, stage ^ 1);
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                    dequant_half(1, 0);
+                    if (step + 1 < step1) load_weights(step + 1);
+                    arrive_ready(3);
+                    phase ^= 1u;
+                }
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                if (step1 > step0) {
+                    wait_mma(0, phase ^ 1u);
+                    wait_mma(1, phase ^ 1u);
+                }
+            } else if (cta_rank == 0) {
+                for (int step = step0; step < step1; ++step) {
+                    const int stage = (step - step0) & 1;
+                    wait_ready(2, phase);
+                    issue_mma(step, stage, 0);
+                    wait_ready(3, phase);
+                    issue_mma(step, stage, 1);
+                    phase ^= 1u;
+                }
             }
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            if (step1 > step0) {
-                wait_mma(0, phase ^ 1u);
-                wait_mma(1, phase ^ 1u);
-            }
-        } else if (cta_rank == 0) {
-            for (int step = step0; step < step1; ++step) {
-                const int stage = (step - step0) & 1;
-                wait_ready(2, phase);
-                issue_mma(step, stage, 0);
-                wait_ready(3, phase);
-                issue_mma(step, stage, 1);
-                phase ^= 1u;
-            }
-        }
         }
     } else {
         if (step0 < step1) copy_x(step0, 0);
