@@ -26,7 +26,8 @@ CASES = [(2, 300, 1024, 9), (2, 512, 1024, 16), (3, 300, 1536, 40), (2, 256, 512
          (1, 130, 640, 65), (2, 4096, 4096, 128), (3, 512, 4096, 700),
          (2, 4096, 512, 2560),      # 160 tiles: whole rounds plus a K-split tail stripe
          # an even number of 256-token tiles and enough weight tiles: the shapes a CTA pair would take
-         (2, 4096, 1024, 512), (3, 4000, 1024, 500), (4, 8192, 1024, 300), (1, 4096, 1536, 1024)]
+         (2, 4096, 1024, 512), (3, 4000, 1024, 500), (4, 8192, 1024, 300), (1, 4096, 1536, 1024),
+         (2, 8192, 640, 512), (3, 20000, 128, 512)]      # the same with K ending inside a 512-column chunk / a single K step
 
 
 @pytest.mark.parametrize("q,N,K,M", CASES)
