@@ -51,10 +51,11 @@ def test_tensor_core_path_matches_oracle(q, N, K, M):
     assert hlq.rel_fro_error(y32, ylut) <= TOL
 
 
-def test_tensor_core_path_terms_and_accumulate():
-    q, G, N, K, M = 2, 128, 300, 1024, 96
-    layer = workloads.hlq_layer(31, "mma/flags", q, G, N, K)
-    X = synth.activations(31, "mma/flags/x", M, K)
+@pytest.mark.parametrize("N,K,M", [(300, 1024, 96), (4096, 1024, 512)])     # one token tile; CTA pairs
+def test_tensor_core_path_terms_and_accumulate(N, K, M):
+    q, G = 2, 128
+    layer = workloads.hlq_layer(31, f"mma/flags/{N}", q, G, N, K)
+    X = synth.activations(31, f"mma/flags/x/{M}", M, K)
     packed = pack_layer(layer)
     ys = gemm_f32(X, packed, N, K, elutq.FLAG_SKIP_OFFSET)
     yb = gemm_f32(X, packed, N, K, elutq.FLAG_OFFSET_ONLY)
