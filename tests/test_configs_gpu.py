@@ -1,6 +1,6 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (C-ABI calls on a
 stream, library-owned scratch): every shape of configs 0, 1 and 3 at M = 1, and the small-batch sweep's
-extremes on one 8B shape.  The 8B shapes are compared in full against the fp64 oracle; the 70B shapes on
+extremes on one 8B shape, and four calls of the prefill configuration.  The 8B shapes at M = 1 are compared in full against the fp64 oracle; the 70B shapes on
 a seeded sample of output rows (first and last tiles plus random rows), which the oracle computes row by row.
 """
 
@@ -64,6 +64,23 @@ def test_config2_small_batch_extremes_on_gate_up(M):
     rows = np.unique(np.concatenate([np.arange(16), np.arange(call.N - 16, call.N), rng.integers(0, call.N, 2048)]))
     ref = hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
     assert hlq.rel_fro_error(y[:, rows], ref) <= TOL_F16
+
+
+@pytest.mark.parametrize("name,M", [("gate_up", 2048), ("down", 2048), ("qkv", 512), ("o", 128)])
+def test_config4_prefill_shapes_sampled(name, M):
+    """The prefill configuration at full size (tensor-core path; CTA pairs for M = 512 and 2048, whole rounds plus
+    the K-split tail stripe on gate_up): sampled weight rows x sampled tokens against the oracle."""
+    call = [c for c in workloads.config4_prefill_calls() if c.name == name and c.M == M][0]
+    layer, X, y = _run(call)
+    rng = np.random.default_rng(7)
+    rows = np.unique(np.concatenate([np.arange(32), np.arange(call.N - 32, call.N), rng.integers(0, call.N, 1024)]))
+    toks = np.unique(np.concatenate([np.arange(8), np.arange(call.M - 8, call.M), rng.integers(0, call.M, 112)]))
+    ref = hlq.matmul(X[toks], layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
+    got = y[np.ix_(toks, rows)]
+    assert np.all(np.isfinite(y))
+    assert hlq.rel_fro_error(got, ref) <= TOL_F16
+    assert max(hlq.rel_fro_error(got[i], ref[i]) for i in range(len(toks))) <= 2 * TOL_F16
+    assert elutq.elutq_device_status() == 0
 
 
 def test_smoke_entry_runs():
