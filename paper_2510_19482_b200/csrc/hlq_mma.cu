@@ -375,8 +375,9 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     auto dequant_half = [&](int hb, int wt) { dequant_half_to(hb, sW + wt * W_BYTES + hb * W_HALF_BYTES); };
 
     // MMAs of one half step (64 k = 4 slices per token tile), issued by one thread; completion arrives on barrier hb.
+    // (Single-CTA schedules; the pair form issues its own in the ring loop below.)
     auto issue_mma = [&](int step, int stage, int hb) {
-        if (tid != (WS ? kMmaThreads : 0) || cta_rank != 0) return;
+        if (tid != (WS ? kMmaThreads : 0)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int tt = 0; tt < TT; ++tt) {
@@ -385,26 +386,14 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 const uint64_t da = desc_swizzle128(x_addr + stage * X_STAGE_BYTES + tt * kXTileBytes + hb * (kTileM * 128) + kk * 32);
                 const uint64_t db = desc_noswizzle(w_addr + hb * W_HALF_BYTES + kk * 256);
                 const uint32_t accumulate = (step != step0 || hb != 0 || kk != 0) ? 1u : 0u;
-                if constexpr (CG == 2) {
-                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
-                                 : "memory");
-                } else {
-                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-                                 :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
-                                 : "memory");
-                }
+                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                             :: "r"(tmem_d + (uint32_t)(tt * NW)), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+                             : "memory");
             }
         }
-        if constexpr (CG == 2) {     // completion arrives on the same barrier of both CTAs of the pair
-            asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                         :: "r"(bar_addr + 8u * hb), "h"((unsigned short)3) : "memory");
-        } else {
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                         :: "r"(bar_addr + 8u * hb) : "memory");
-        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     :: "r"(bar_addr + 8u * hb) : "memory");
     };
     auto publish = [&]() {     // generic-proxy writes of this thread -> visible to the tensor core, then CTA barrier
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -577,7 +566,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                     wait_mma(0, phase ^ 1u);
                     wait_mma(1, phase ^ 1u);
                 }
-            } else if (cta_rank == 0) {
+            } else {
                 for (int step = step0; step < step1; ++step) {
                     const int stage = (step - step0) & 1;
                     wait_ready(2, phase);
