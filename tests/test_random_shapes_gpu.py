@@ -42,3 +42,32 @@ def test_random_shape(i, q, G, N, K, M):
         ylut = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)
         assert hlq.rel_fro_error(ylut, ref) <= 5e-6
     assert elutq.elutq_device_status() == 0
+
+
+def _prefill_cases():
+    rng = np.random.default_rng(20251020)
+    out = []
+    for i in range(20):
+        q = int(rng.integers(1, 5))
+        K = 128 * int(rng.integers(1, 25))
+        N = int(rng.choice([2048, 3000, 4096, 5000, 8192]))
+        M = int(rng.choice([257, 300, 512, 513, 700, 1000, 1024, 1500, 2048]))
+        out.append((i, q, N, K, M))
+    return out
+
+
+@pytest.mark.parametrize("i,q,N,K,M", _prefill_cases())
+def test_random_prefill_shape(i, q, N, K, M):
+    """Prefill-sized batches at G = 128: several token tiles per weight tile (CTA pairs when their number is even),
+    K splits, tail stripes, ragged N / M / K."""
+    G = 128
+    layer = workloads.hlq_layer(80 + i, f"randp/{i}", q, G, N, K, signed_scales=(i % 3 == 0))
+    X = synth.activations(80 + i, f"randp/x/{i}", M, K, outliers=(i % 4 == 0))
+    packed = pack_layer(layer)
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    y16 = gemm_f16(X, packed, N, K)
+    assert np.all(np.isfinite(y16))
+    assert hlq.rel_fro_error(y16, ref) <= 1e-3
+    rows = range(0, M, max(1, M // 32))
+    assert max(hlq.rel_fro_error(y16[m], ref[m]) for m in rows) <= 2e-3
+    assert elutq.elutq_device_status() == 0
