@@ -218,6 +218,66 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
 int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
 
 /*
+ * A decode step as one launch (Appendix B's procedure at M = 1, call after call).
+ *
+ * At M = 1 every linear of a decode step is one bit-serial LUT GEMV; launched one by one, each pays its own
+ * kernel start, K-split reduction and kernel end, during which HBM idles.  A chain runs a fixed list of
+ * such calls - typically all linears of a decode step, in model order - in ONE persistent launch (one per run
+ * of consecutive calls with equal (q, G): a model has one such pair, a mixed list is cut at the changes):
+ * Y_c[N_c] = X_c[K_c] * W_hat_c^T for c = 0 .. n_calls-1, each result identical in value to elutq_lut_gemm
+ * up to the order of the fp32 K-chunk sum (chunks are always added in ascending order, so a chain is
+ * bit-reproducible from launch to launch).
+ *
+ * Ordering: the results are those of the calls run one after another in list order.  The plan derives from
+ * the buffer addresses which earlier calls a call really depends on - its X or Y overlaps their Y, or its Y
+ * their X - and the launch waits exactly for those; calls whose buffers are disjoint overlap freely (a
+ * decode step whose linears read separately produced activations streams without a pause, a chain in which
+ * Y of one call is X of the next is run strictly in turn).
+ *
+ *   elutq_chain_plan_bytes  size of the plan buffer for a list (pure function, no CUDA call)
+ *   elutq_chain_plan        validates the list, reads q and G of every blob (elutq_describe's rules) and
+ *                           writes the plan into `plan`: caller-owned DEVICE memory, 256-byte aligned, of
+ *                           at least that size.  It holds the descriptors, the K-split scratch and the
+ *                           hand-over counters.  Synchronises `stream`; an offline step, once per list.
+ *                           Pointers and shapes are frozen in the plan; the buffers they name may change
+ *                           content between runs.  M is 1; flags per call: ELUTQ_FLAG_OUT_F32,
+ *                           ELUTQ_FLAG_ACCUMULATE (others: ELUTQ_ERR_UNSUPPORTED).
+ *   elutq_chain_run         one cooperative launch on `stream` (one CTA per SM; the device must be able to
+ *                           hold them all at once, else ELUTQ_ERR_CUDA and nothing runs).  Allocates
+ *                           nothing.  Runs of one plan must not overlap on the GPU.  Every CTA first
+ *                           compares each blob's header with the plan; on a mismatch the launch ends at
+ *                           once with status 0x7C0B and no tile is read.
+ *   elutq_chain_run_opts    the same with explicit tuning values (test / measurement entry): the poll
+ *                           limit of the hand-over waits (0 = default, 2^22), the number of items per warp
+ *                           requested from L2 ahead of each call (0..8, default 2) and whether a rolling
+ *                           L2 prefetch runs two items ahead of the register loads (0/1, default 1).
+ *   elutq_chain_status      synchronises `stream` and reads the plan's status word: 0, or 0x7C05 after a
+ *                           hand-over wait ran out (every wait is a bounded poll; the launch then finishes
+ *                           without waiting any further and its results are undefined), or 0x7C0B.  After a
+ *                           non-zero status the plan must be written again with elutq_chain_plan.
+ */
+typedef struct elutq_gemv_call {
+    const void* X;        /* device fp16 [K]                                   */
+    const void* packed;   /* device blob of elutq_pack for (N, K)              */
+    void* Y;              /* device fp16 [N] (float [N] with ELUTQ_FLAG_OUT_F32) */
+    int N, K;
+    unsigned flags;
+} elutq_gemv_call;
+
+#define ELUTQ_CHAIN_MAX_CALLS 4096
+
+int elutq_chain_plan_bytes(const elutq_gemv_call* calls, int n_calls, size_t* bytes);
+int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size_t plan_bytes, void* stream);
+int elutq_chain_run(void* plan, int n_calls, void* stream);
+int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefetch_first, int prefetch_ahead,
+                         void* stream);
+int elutq_chain_status(const void* plan, void* stream, int* status);
+/* The library keeps a small host-side note per planned buffer (which runs of equal (q, G) to launch);
+ * elutq_chain_run returns ELUTQ_ERR_SHAPE for a buffer that this process has not planned.  Call this before
+ * freeing a plan buffer. */
+int elutq_chain_forget(const void* plan);
+
+/*
  * Algorithm 1 (Section 4.2): alternating optimisation of the HLQ parameters, the offline step that
  * produces what elutq_pack consumes.  For every group of G consecutive weights of a row: uniform
  * initialisation (Delta = (max - min) / (2^q - 1), s = [Delta, 2 Delta, ...], z = min), then t_max

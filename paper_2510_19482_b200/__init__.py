@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     FLAG_LUT_ONLY,
     FLAG_TABLE_F16,
     FLAG_TABLE_I8,
+    GemvCall,
     lib,
     library_path,
     elutq_packed_bytes,
@@ -33,6 +34,12 @@ from .binding import (  # noqa: F401
     elutq_lut_gemm_host,
     elutq_lut_gemm_static,
     elutq_hlq_fit,
+    elutq_chain_plan_bytes,
+    elutq_chain_plan,
+    elutq_chain_run,
+    elutq_chain_run_opts,
+    elutq_chain_status,
+    elutq_chain_forget,
     elutq_device_status,
     elutq_launch_count,
     elutq_release_scratch,

@@ -21,6 +21,11 @@ FLAG_TABLE_F16 = 0x100
 FLAG_TABLE_I8 = 0x200
 
 
+class GemvCall(ctypes.Structure):
+    """elutq_gemv_call: one M = 1 call of a chain."""
+    _fields_ = [("X", c_void_p), ("packed", c_void_p), ("Y", c_void_p), ("N", c_int), ("K", c_int), ("flags", c_uint)]
+
+
 class ElutqError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -50,6 +55,12 @@ _SIGNATURES = {
     "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_lut_gemm_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_hlq_fit": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "elutq_chain_plan_bytes": (c_int, [ctypes.POINTER(GemvCall), c_int, ctypes.POINTER(c_size_t)]),
+    "elutq_chain_plan": (c_int, [ctypes.POINTER(GemvCall), c_int, c_void_p, c_size_t, c_void_p]),
+    "elutq_chain_run": (c_int, [c_void_p, c_int, c_void_p]),
+    "elutq_chain_run_opts": (c_int, [c_void_p, c_int, c_uint, c_int, c_int, c_void_p]),
+    "elutq_chain_status": (c_int, [c_void_p, c_void_p, ctypes.POINTER(c_int)]),
+    "elutq_chain_forget": (c_int, [c_void_p]),
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
@@ -197,3 +208,50 @@ def elutq_device_status(stream=None) -> int:
     out = c_int(0)
     _check(lib().elutq_device_status(_stream(stream), ctypes.byref(out)), "elutq_device_status")
     return out.value
+
+
+def _call_array(calls):
+    """calls: sequence of (X, packed, Y, N, K[, flags]) with tensors or raw addresses -> ctypes array."""
+    arr = (GemvCall * len(calls))()
+    for i, c in enumerate(calls):
+        X, packed, Y, N, K = c[:5]
+        flags = c[5] if len(c) > 5 else 0
+        arr[i] = GemvCall(X if isinstance(X, int) else _ptr(X), packed if isinstance(packed, int) else _ptr(packed),
+                          Y if isinstance(Y, int) else _ptr(Y), N, K, flags)
+    return arr
+
+
+def elutq_chain_plan_bytes(calls) -> int:
+    out = c_size_t(0)
+    _check(lib().elutq_chain_plan_bytes(_call_array(calls), len(calls), ctypes.byref(out)), "elutq_chain_plan_bytes")
+    return out.value
+
+
+def elutq_chain_plan(calls, plan=None, stream=None):
+    """Writes the plan of a list of M = 1 calls into a device buffer (allocated here when not given); returns it."""
+    import torch
+    if plan is None:
+        plan = torch.empty(elutq_chain_plan_bytes(calls), dtype=torch.uint8, device="cuda")
+    _check(lib().elutq_chain_plan(_call_array(calls), len(calls), _ptr(plan), plan.numel() * plan.element_size(),
+                                  _stream(stream)), "elutq_chain_plan")
+    return plan
+
+
+def elutq_chain_run(plan, n_calls: int, stream=None) -> None:
+    _check(lib().elutq_chain_run(_ptr(plan), n_calls, _stream(stream)), "elutq_chain_run")
+
+
+def elutq_chain_run_opts(plan, n_calls: int, wait_limit: int = 0, prefetch_first: int = 2, prefetch_ahead: int = 1,
+                         stream=None) -> None:
+    _check(lib().elutq_chain_run_opts(_ptr(plan), n_calls, wait_limit, prefetch_first, prefetch_ahead, _stream(stream)),
+           "elutq_chain_run_opts")
+
+
+def elutq_chain_status(plan, stream=None) -> int:
+    out = c_int(0)
+    _check(lib().elutq_chain_status(_ptr(plan), _stream(stream), ctypes.byref(out)), "elutq_chain_status")
+    return out.value
+
+
+def elutq_chain_forget(plan) -> None:
+    _check(lib().elutq_chain_forget(_ptr(plan)), "elutq_chain_forget")

@@ -8,7 +8,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["api.cu", "pack.cu", "lut_gemv.cu", "lut_gemm.cu", "hlq_mma.cu", "hlq_fit.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "pack.cu", "lut_gemv.cu", "lut_gemm.cu", "hlq_mma.cu", "hlq_fit.cu", "static_scratch.cu", "lut_chain.cu"]
 LIB = os.path.join(HERE, "libelutq.so")
 
 
@@ -23,7 +23,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu under csrc/ into libelutq.so; returns the library path."""
     csrc = os.path.join(HERE, "csrc")
     srcs = [os.path.join(csrc, s) for s in SOURCES]
-    deps = srcs + [os.path.join(csrc, "common.cuh"), os.path.join(ROOT, "include", "elutq.h")]
+    deps = srcs + [os.path.join(csrc, "common.cuh"), os.path.join(csrc, "lut_core.cuh"), os.path.join(ROOT, "include", "elutq.h")]
     if not force and not _newer_than_lib(deps):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")

@@ -152,7 +152,7 @@ int launch_copy_in(const void* src, void* dst, size_t bytes, cudaStream_t stream
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
+    cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, copy_in_kernel, reinterpret_cast<const uint8_t*>(src), reinterpret_cast<uint8_t*>(dst), bytes);
     count_launch(1);
     return (int)e;
@@ -202,7 +202,7 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY |
                                   ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8;
     if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
-    else if (M >= (debug_env("ELUTQ_DEBUG_MMA_MIN_M") > 0 ? debug_env("ELUTQ_DEBUG_MMA_MIN_M") : ELUTQ_TENSOR_MIN_M) && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
+    else if (M >= ELUTQ_TENSOR_MIN_M && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
     else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);
     if (ce != 0) return cuda_fail((cudaError_t)ce);
     return ELUTQ_OK;
@@ -350,7 +350,7 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host, in
     const bool small = xb + yb <= ((size_t)1 << 20);
     const void* x_map = small ? host_device_pointer(X_host) : nullptr;
     void* y_map = small ? const_cast<void*>(host_device_pointer(Y_host)) : nullptr;
-    if (x_map && y_map && aligned(x_map, 16) && aligned(y_map, 16) && debug_env("ELUTQ_DEBUG_HOST_MEMCPY") == 0) {
+    if (x_map && y_map && aligned(x_map, 16) && aligned(y_map, 16)) {
         int ce = launch_copy_in(x_map, xd, xb, (cudaStream_t)stream);
         if (ce != 0) return cuda_fail((cudaError_t)ce);
         return run_gemm(xd, packed, y_map, M, N, K, 0u, nullptr, 0, true, stream);

@@ -52,7 +52,7 @@ struct GemmArgs {
     const uint8_t* tiles;    // packed + header
     void* Y;                 // fp16 or fp32 [M][N]
     float* partials;         // [n_kc][M][n_rb*16] (unused when n_kc == 1)
-    unsigned* counters;      // [n_rb * ceil(M/MB)] arrival counters, zero between calls
+    unsigned* counters;      // control words of the scratch (may be null): word 0 = device status (0 = fine)
     int M, N, K;
     int n_rb, n_kc;
     unsigned flags;
@@ -62,7 +62,6 @@ struct GemmArgs {
                              // partition of the item list); range r holds rb_q (+1 if r < rb_r) row blocks;
                              // CTA b = group * ranges + r, group = `cpc` consecutive chunks
     int cpc;                 // chunks per CTA in the aligned partition
-    int fused_reduce;        // 1: the last CTA of a range reduces it in-kernel (needs counters); 0: finalize kernel
     int cluster_reduce;      // 1: launched as clusters of n_kc CTAs (one per chunk, same row range): partials stay in
                              //    shared memory and are reduced through distributed shared memory
 };
@@ -78,7 +77,6 @@ int launch_hlq_mma(const GemmArgs& a, int q, int G, int num_sms, cudaStream_t st
 
 // col0 / cols restrict the reduction to output columns [col0, col0 + cols) (cols = 0: all N columns).
 int launch_finalize(const GemmArgs& a, int n_chunks, bool pdl, cudaStream_t stream, int col0 = 0, int cols = 0);
-int debug_env(const char* name);
 void count_launch(unsigned n = 1);
 
 // api.cu helpers shared with other translation units: blob description (registry or header read),
@@ -158,6 +156,24 @@ __device__ __forceinline__ float ld_cluster_f32(const float* local_smem_ptr, uns
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
     return v;
 }
+// Device status codes (word 0 of the control area; read back by elutq_device_status / elutq_chain_status).
+constexpr unsigned kStatusWaitExpired = 0x7C05u;    // a bounded wait ran out
+constexpr unsigned kStatusBlobMismatch = 0x7C0Bu;   // the blob header does not describe what the kernel was launched for
+
+// Every GEMM kernel compares the header of the blob it was handed with the geometry it was launched for before it
+// reads any tile: a stale description of an address that now holds another blob must never turn into reads
+// past the end of the buffer.  `tiles` points just behind the 128-byte header.  On mismatch the status word is
+// raised and the caller returns without touching the tiles (every thread sees the same header, so a CTA
+// leaves as a whole).
+__device__ __forceinline__ bool blob_header_matches(const uint8_t* tiles, int q, int G, int N, int K, unsigned* status) {
+    const uint4 h0 = __ldg(reinterpret_cast<const uint4*>(tiles - ELUTQ_HEADER_BYTES));
+    const uint2 h1 = __ldg(reinterpret_cast<const uint2*>(tiles - ELUTQ_HEADER_BYTES + 16));
+    const bool ok = h0.x == (uint32_t)kMagic && h0.y == (uint32_t)kVersion && h0.z == (uint32_t)q && h0.w == (uint32_t)G &&
+                    h1.x == (uint32_t)N && h1.y == (uint32_t)K;
+    if (!ok && status != nullptr && threadIdx.x == 0) atomicExch(status, kStatusBlobMismatch);
+    return ok;
+}
+
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -664,7 +664,7 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     const int n_tiles = (a.N + NW - 1) / NW, m_tiles = (a.M + TT * kTileM - 1) / (TT * kTileM);
     const long long tiles = (long long)n_tiles * m_tiles;
     const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;   // the partial buffer holds 2 * n_kc slices
-    const bool pdl = debug_env("ELUTQ_DEBUG_NO_PDL") == 0;
+    const bool pdl = true;
 
     auto launch = [&](int n_tile0, int n_count, int splits) -> cudaError_t {
         cudaLaunchConfig_t cfg = {};
@@ -691,7 +691,7 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     };
 
     // Fewer tiles than SMs: K split while the tile count leaves SMs idle (partials cost M*N*4 bytes per split).
-    if (tiles <= num_sms || debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0 || debug_env("ELUTQ_DEBUG_MMA_NO_TAIL") > 0) {
+    if (tiles <= num_sms) {
         int splits = 1;
         while (splits * 2 <= max_splits && tiles * splits * 2 <= (long long)num_sms) splits *= 2;
         {   // a split that is no power of two (uneven step counts per CTA) only where it adds 30 % more CTAs or more
@@ -702,7 +702,6 @@ int launch_mma_cfg(const GemmArgs& a, int num_sms, cudaStream_t stream) {
             if (any > 4 * a.n_kc) any = 4 * a.n_kc;
             if (any * 10 >= (long long)splits * 13) splits = (int)any;
         }
-        if (debug_env("ELUTQ_DEBUG_MMA_SPLITS") > 0) splits = debug_env("ELUTQ_DEBUG_MMA_SPLITS");
         if (splits > max_splits) splits = max_splits;
         cudaError_t e = launch(0, n_tiles, splits);
         if (e != cudaSuccess || splits == 1) return (int)e;
@@ -734,18 +733,16 @@ template <int Q>
 int launch_mma_q(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     // Two token tiles per CTA once M exceeds one tile; 256 weight rows per CTA unless even the largest K split
     // would leave most SMs without work.
-    const bool two = a.M > kTileM && debug_env("ELUTQ_DEBUG_MMA_TT") != 1;
+    const bool two = a.M > kTileM;
     const long long m_tiles = two ? (a.M + 2 * kTileM - 1) / (2 * kTileM) : (a.M + kTileM - 1) / kTileM;
     const long long tiles256 = (long long)((a.N + 255) / 256) * m_tiles;
     const int max_splits = 2 * a.n_kc < 16 ? 2 * a.n_kc : 16;
     bool narrow = tiles256 * max_splits * 2 <= num_sms;
-    if (debug_env("ELUTQ_DEBUG_MMA_NW") == 128) narrow = true;
-    if (debug_env("ELUTQ_DEBUG_MMA_NW") == 256) narrow = false;
     // measured: the warp-specialised form is 3-5 % faster (no CTA-wide barrier in the step, the issuing thread dequantises nothing)
     // measured: a CTA pair per weight tile (each CTA dequantises half of it) is 8-22 % faster again; it needs an even
     // number of 256-token tiles
-    if (two && !narrow && m_tiles % 2 == 0 && debug_env("ELUTQ_DEBUG_MMA_NO_PAIR") == 0) return launch_mma_cfg<Q, 256, 2, true, 2>(a, num_sms, stream);
-    if (two && !narrow && debug_env("ELUTQ_DEBUG_MMA_NO_WS") == 0) return launch_mma_cfg<Q, 256, 2, true>(a, num_sms, stream);
+    if (two && !narrow && m_tiles % 2 == 0) return launch_mma_cfg<Q, 256, 2, true, 2>(a, num_sms, stream);
+    if (two && !narrow) return launch_mma_cfg<Q, 256, 2, true>(a, num_sms, stream);
     if (two) return narrow ? launch_mma_cfg<Q, 128, 2>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 2>(a, num_sms, stream);
     return narrow ? launch_mma_cfg<Q, 128, 1>(a, num_sms, stream) : launch_mma_cfg<Q, 256, 1>(a, num_sms, stream);
 }

@@ -1,0 +1,741 @@
+// A list of M = 1 decode calls run by persistent launches (elutq_chain_plan / elutq_chain_run).
+//
+// A decode step is a fixed sequence of linears on one stream.  Launched one by one, every call pays its own
+// chain of cross-SM hand-overs (kernel start, activation load, table build, K-split reduction, kernel end), during
+// which HBM idles; for the 8B layer shapes that chain is several times longer than the time the call's bytes need.
+// Here one cooperative grid (one 1024-thread CTA per SM) walks a run of consecutive calls that share (q, G) - a
+// model has one such pair, so normally the whole list is one launch; a list that mixes them is cut into one
+// launch per run.  Inside a CTA the warps are specialised (Appendix B's two phases run side by side):
+//
+//   * 4 builder warps load the activations of the CTA's next K chunk and fill the other of two table buffers
+//     (fused 8-bit tables, 64 KiB each) while
+//   * 28 look-up warps stream the packed weights of the current chunk (one warp per 16-row x 512-column item,
+//     registers refilled one item ahead, as in lut_gemv.cu) and sum table entries.  Buffers are handed over through
+//     shared-memory mbarriers ("full" / "free" per buffer).
+//   * K-split: every partial sum is stored together with a tag (launch epoch and call number) in one 8-byte
+//     word.  The CTAs that share a row range split its rows among themselves; the builder warps poll (bounded)
+//     the tagged words of their rows, add the chunks in ascending order - bit-reproducible - and write Y.  No
+//     fence, no ticket, no second kernel: the load that finds the tag is the load that brings the value.
+//   * Ordering: the result is what the calls give when run one after another.  The plan records, from the buffer
+//     addresses, which earlier calls a call really depends on (its X or Y overlaps their Y, or its Y their X);
+//     before the builders read X they wait (bounded) for the completion counters of exactly those calls.  Calls
+//     without such a dependency overlap freely, so HBM keeps streaming across call boundaries.
+//   * The builders also ask L2 for the look-up warps' first items of the next call (cp.async.bulk.prefetch.L2)
+//     a whole call ahead, and a rolling prefetch runs two items ahead of the register loads.
+//
+// Every wait is a bounded poll; when one runs out the CTA raises the plan's status word, stops waiting for
+// the rest of the launch (results are then undefined) and returns normally.
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <vector>
+
+#include "lut_core.cuh"
+
+namespace elutq {
+
+namespace {
+
+constexpr unsigned kChainMagic = 0x4E494843u;
+constexpr int kChainRegions = 3;              // scratch regions for the tagged partial sums, used round-robin
+constexpr int kDescSlots = 4;
+constexpr int kLookupWarps = 26;
+constexpr int kBuilderWarps = 4;
+constexpr int kFinisherWarps = kGemvWarps - kLookupWarps - kBuilderWarps;
+constexpr int kBuilderThreads = kBuilderWarps * 32;
+constexpr int kFinisherThreads = kFinisherWarps * 32;
+// shared memory: two table buffers, then per buffer 16 group sums, four mbarriers, flags, descriptor ring
+constexpr int kOffGsum = 2 * kTableBytes;
+constexpr int kOffBar = kOffGsum + 128;
+constexpr int kOffShared = kOffBar + 32;
+constexpr int kOffDesc = kOffGsum + 256;                  // builders' descriptor ring
+constexpr int kOffWarpDesc = kOffDesc + kDescSlots * 128;   // look-up and finisher warps: two descriptor slots per warp
+constexpr int kChainSmem = kOffWarpDesc + (kLookupWarps + kFinisherWarps) * 2 * 128;
+constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
+constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
+
+struct ChainCtl {                             // first 256 bytes of a plan
+    unsigned magic, n_calls, status, epoch;
+    unsigned exit_ticket, grid, reserved0, reserved1;
+    unsigned long long done_off, calls_off, slots_off, region_bytes, total_bytes;
+};
+
+struct ChainCall {                            // 128 bytes
+    const __half* X;
+    const uint8_t* tiles;                     // packed + header
+    void* Y;
+    unsigned long long* slots;                // [n_kc][n_rb * 16] tagged partial sums of this call's scratch region
+    int N, K, n_rb, n_kc;
+    int q, G;
+    unsigned flags;
+    int dep_first, dep_last;                  // earlier calls whose completion must precede reading X / writing Y
+                                              // (dep_first > dep_last: none)
+    int ranges, rb_q, rb_r, cpc;
+    int groups, n_ctas;
+    int guard_call;                           // call that used this scratch region last (-1: none): it must be complete
+    unsigned done_target;                     // completion reports per launch: one per CTA (one per look-up warp of every
+                                              // CTA when the call has no K split)
+    int pad[7];
+};
+static_assert(sizeof(ChainCall) == 128, "descriptor size");
+static_assert(sizeof(ChainCtl) <= 256, "control block size");
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2_line(const void* p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void bar_builders() {          // named barrier 1: the builder warps only
+    asm volatile("bar.sync 1, %0;" ::"n"(kBuilderThreads) : "memory");
+}
+__device__ __forceinline__ void bar_finishers() {         // named barrier 2: the finisher warps only
+    asm volatile("bar.sync 2, %0;" ::"n"(kFinisherThreads) : "memory");
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"((uint32_t)__cvta_generic_to_shared(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+struct ChainShared {
+    volatile int abort;                       // a wait ran out: stop waiting
+    unsigned epoch;
+};
+
+extern __shared__ __align__(1024) uint8_t chain_smem[];
+
+__device__ __forceinline__ ChainShared* chain_shared() { return reinterpret_cast<ChainShared*>(chain_smem + kOffShared); }
+__device__ __forceinline__ ChainCall* chain_desc(int c) {
+    return reinterpret_cast<ChainCall*>(chain_smem + kOffDesc) + (c & (kDescSlots - 1));
+}
+__device__ __forceinline__ ChainCall* warp_desc(int lw, int c) {
+    return reinterpret_cast<ChainCall*>(chain_smem + kOffWarpDesc) + lw * 2 + (c & 1);
+}
+__device__ __forceinline__ uint64_t* bar_full(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + b; }
+__device__ __forceinline__ uint64_t* bar_free(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + 2 + b; }
+
+__device__ __forceinline__ void raise_abort(unsigned* status) {
+    ChainShared* sh = chain_shared();
+    if (!sh->abort) {
+        sh->abort = 1;
+        atomicExch(status, kStatusWaitExpired);
+    }
+}
+// Bounded wait on a shared-memory barrier phase.
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, unsigned* status) {
+    ChainShared* sh = chain_shared();
+    for (unsigned i = 0; !mbar_test(bar, parity); ++i) {
+        if (i >= limit || sh->abort) {
+            raise_abort(status);
+            return;
+        }
+    }
+}
+// Bounded poll: true once *p has reached `target` (wrap-safe comparison).
+__device__ __forceinline__ bool wait_reached(const unsigned* p, unsigned target, unsigned limit) {
+    for (unsigned i = 0; i < limit; ++i) {
+        if ((int)(ld_acquire_u32(p) - target) >= 0) return true;
+        if (i > 64) __nanosleep(64);
+    }
+    return false;
+}
+
+__device__ __forceinline__ void chain_store(void* Y, unsigned flags, size_t idx, float y) {
+    if (flags & ELUTQ_FLAG_OUT_F32) {
+        float* Yf = reinterpret_cast<float*>(Y);
+        Yf[idx] = (flags & ELUTQ_FLAG_ACCUMULATE) ? __ldcg(Yf + idx) + y : y;
+    } else {
+        __half* Yh = reinterpret_cast<__half*>(Y);
+        if (flags & ELUTQ_FLAG_ACCUMULATE) y += __half2float(__ldcg(reinterpret_cast<const __half*>(Yh) + idx));
+        Yh[idx] = __float2half_rn(y);
+    }
+}
+
+// Row range and chunk group of CTA `bid` in call d.
+struct ChainPart {
+    int rb0, rb1, kc0, nseg, grp;
+};
+__device__ __forceinline__ ChainPart chain_part(const ChainCall* d, int bid) {
+    ChainPart p;
+    p.grp = bid / d->ranges;
+    const int range = bid - p.grp * d->ranges;
+    p.rb0 = range * d->rb_q + min(range, d->rb_r);
+    p.rb1 = p.rb0 + d->rb_q + (range < d->rb_r ? 1 : 0);
+    p.kc0 = p.grp * d->cpc;
+    p.nseg = min(d->cpc, d->n_kc - p.kc0);
+    return p;
+}
+
+// K-split reduction of call d by this CTA's builder threads: the `groups` CTAs of a row range split its rows;
+// every thread polls the tagged partial sums of its row (all chunks), adds them in ascending chunk order and
+// writes Y.
+__device__ __noinline__ void chain_reduce(const ChainCall* d, const ChainPart p, unsigned tag, unsigned limit,
+                                          unsigned* status, int ft) {
+    ChainShared* sh = chain_shared();
+    const int rows = min(p.rb1 * kTileRows, d->N) - p.rb0 * kTileRows;
+    const int per = (rows + d->groups - 1) / d->groups;
+    const int r0 = p.rb0 * kTileRows + p.grp * per;
+    const int r1 = min(p.rb0 * kTileRows + rows, r0 + per);
+    const size_t n_pad = (size_t)d->n_rb * kTileRows;
+    const int n_kc = d->n_kc;
+    for (int row = r0 + ft; row < r1; row += kFinisherThreads) {
+        const unsigned long long* src = d->slots + row;
+        float sum = 0.f;
+        for (int c0 = 0; c0 < n_kc; c0 += 8) {
+            unsigned long long v[8];
+            bool ok = false;
+            for (unsigned spin = 0; !ok; ++spin) {
+                ok = true;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (c0 + i < n_kc) {
+                        v[i] = ld_relaxed_u64(src + (size_t)(c0 + i) * n_pad);
+                        ok = ok && (unsigned)(v[i] >> 32) == tag;
+                    }
+                }
+                if (!ok && (spin >= limit || sh->abort)) {
+                    raise_abort(status);
+                    break;
+                }
+                if (!ok && spin > 64) __nanosleep(64);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (c0 + i < n_kc) sum += __uint_as_float((unsigned)v[i]);
+        }
+        chain_store(d->Y, d->flags, (size_t)row, sum);
+    }
+}
+
+// Fused tables of chunk kc (and its group sums) built by the builder warps: lane -> column pair (2*lane,
+// 2*lane+1) as in build_tables; builder warp bw takes the (high nibble, low-nibble half) combinations
+// vw = bw, bw + 4, ... of the 32 that a full CTA would spread over its warps.
+template <int G>
+__device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const __half* __restrict__ X, int kc, int K,
+                                                int bw, int lane) {
+    constexpr int W = G / 8;
+    const int k0 = kc * kChunkK + lane * 16;
+    float2 x[8];
+    if (k0 < K) {
+        const uint4 r0 = __ldcg(reinterpret_cast<const uint4*>(X + k0));      // past the incoherent L1: X may have
+        const uint4 r1 = __ldcg(reinterpret_cast<const uint4*>(X + k0 + 8));  // been written during this launch
+        const uint32_t a[4] = {r0.x, r0.y, r0.z, r0.w}, b[4] = {r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&a[i]));
+            const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&b[i]));
+            x[2 * i] = make_float2(fa.x, fb.x);
+            x[2 * i + 1] = make_float2(fa.y, fb.y);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = make_float2(0.f, 0.f);
+    }
+#pragma unroll
+    for (int lh = 0; lh < 2; ++lh) {
+        float2 A[8];
+        A[0] = lh ? x[3] : make_float2(0.f, 0.f);
+        A[1] = fadd2(A[0], x[0]);
+        A[2] = fadd2(A[0], x[1]);
+        A[3] = fadd2(A[1], x[1]);
+        A[4] = fadd2(A[0], x[2]);
+        A[5] = fadd2(A[1], x[2]);
+        A[6] = fadd2(A[2], x[2]);
+        A[7] = fadd2(A[3], x[2]);
+#pragma unroll
+        for (int s = 0; s < 16 / kBuilderWarps; ++s) {
+            const int hi = bw + s * kBuilderWarps;
+            float2 Bv = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                if ((hi >> b) & 1) Bv = fadd2(Bv, x[4 + b]);
+            float2* row = reinterpret_cast<float2*>(tab) + (size_t)(hi * 16 + lh * 8) * 32 + lane;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) row[t * 32] = fadd2(A[t], Bv);
+            if (lh == 1 && hi == 15) {          // entry 255 = sum of the column's 8 activations -> group sums
+                const float2 e = fadd2(A[7], Bv);
+                float total = e.x + e.y;
+#pragma unroll
+                for (int off = W / 4; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+                if ((lane % (W / 2)) == 0) gsum[lane / (W / 2)] = total;
+            }
+        }
+    }
+}
+
+// Items of one chunk (kc) of call d on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of
+// the chunk on entry and its first item of the next chunk (when there is one) on exit.
+template <int Q, int G, int B>
+__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const ChainCall* d, const int rb0,
+                                            const int rb1, const int kc, const bool more_segs, const uint8_t* seg_vp,
+                                            const unsigned tag, const int pf_ahead, const int lw, const int lane) {
+    using C = Cfg<Q, G>;
+    const uint8_t* const tab = chain_smem + B * kTableBytes;
+    const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
+    const int h = lane >> 4, l = lane & 15;
+    float S[C::GL];
+    load_group_sums<G>(S, gsum, h, l, true);
+    const int n_rb = d->n_rb;
+    const uint8_t* next_seg_vp = seg_vp + (size_t)n_rb * C::TILE_BYTES;
+    const uint8_t* vp = seg_vp;
+    unsigned long long* out = d->slots + (size_t)kc * ((size_t)n_rb * kTileRows) + l;
+    for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
+        // next item of this warp: the same chunk, else its first item of the CTA's next chunk
+        const bool in_seg = rb + kLookupWarps < rb1;
+        const uint8_t* nvp = in_seg ? vp + kLookupWarps * C::TILE_BYTES : next_seg_vp;
+        const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
+        if (pf_ahead > 0 && lane == 0 && rb + 2 * kLookupWarps < rb1)   // rolling L2 prefetch, one item beyond the register loads
+            prefetch_l2_bulk(vp + 2 * kLookupWarps * C::TILE_BYTES, C::TILE_BYTES);
+        float y;
+        if (in_seg || more_segs) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
+        else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
+        if (h == 0) {
+            if (d->n_kc == 1) {
+                if (rb * kTileRows + l < d->N) chain_store(d->Y, d->flags, (size_t)(rb * kTileRows + l), y);
+            } else {
+                st_relaxed_u64(out + rb * kTileRows, ((unsigned long long)tag << 32) | __float_as_uint(y));
+            }
+        }
+        vp = nvp;
+    }
+}
+
+// Calls [c_begin, c_end) of the plan, all with the kernel's (Q, G).
+template <int Q, int G>
+__global__ void __launch_bounds__(kGemvThreads, 1)
+lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const int c_begin, const int c_end,
+                 const int last_run, const unsigned spin_limit, const int pf_first, const int pf_ahead) {
+    using C = Cfg<Q, G>;
+    uint8_t* const smem = chain_smem;
+    ChainShared* sh = chain_shared();
+    unsigned* done = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(ctl) + ctl->done_off);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bid = blockIdx.x;
+
+    // Before any tile is read: the plan is the one the host launched, and every blob of this run still carries
+    // the header it was planned with.
+    int bad = (ctl->magic != kChainMagic || ctl->n_calls != (unsigned)n_calls) ? 1 : 0;
+    if (!bad) {
+        for (int c = c_begin + tid; c < c_end; c += kGemvThreads) {
+            const ChainCall* d = calls + c;
+            if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) bad = 1;
+        }
+    }
+    if (tid < 8 * min(c_end - c_begin, 2)) {
+        const int c = c_begin + (tid >> 3);
+        cp_async16(reinterpret_cast<uint8_t*>(chain_desc(c)) + (tid & 7) * 16, reinterpret_cast<const uint8_t*>(calls + c) + (tid & 7) * 16);
+    }
+    if (tid == 0) {
+        sh->abort = 0;
+        sh->epoch = ctl->epoch;
+        mbar_init(bar_full(0), kBuilderThreads);
+        mbar_init(bar_full(1), kBuilderThreads);
+        mbar_init(bar_free(0), kLookupWarps * 32);
+        mbar_init(bar_free(1), kLookupWarps * 32);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    cp_async_wait_all();
+    if (__syncthreads_or(bad)) {
+        if (tid == 0) atomicExch(&ctl->status, kStatusBlobMismatch);
+        return;                               // the same for every CTA: nobody is left waiting
+    }
+    const unsigned epoch = sh->epoch;
+    unsigned* const status = &ctl->status;
+
+    // Per-warp descriptor copies for the warps that run on their own (look-up and finisher warps): the copy of
+    // call c + 1 is fetched while call c is worked on.
+    auto desc_begin = [&](int slot_warp) {
+        if (lane < 8) cp_async16(reinterpret_cast<uint8_t*>(warp_desc(slot_warp, c_begin)) + lane * 16,
+                                 reinterpret_cast<const uint8_t*>(calls + c_begin) + lane * 16);
+    };
+    auto desc_next = [&](int slot_warp, int c) -> const ChainCall* {
+        if (lane < 8) {
+            cp_async_wait_all();
+            if (c + 1 < c_end) {
+                cp_async16(reinterpret_cast<uint8_t*>(warp_desc(slot_warp, c + 1)) + lane * 16,
+                           reinterpret_cast<const uint8_t*>(calls + (c + 1)) + lane * 16);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            }
+        }
+        __syncwarp();
+        return warp_desc(slot_warp, c);
+    };
+
+    if (warp < kLookupWarps) {
+        // ---------------------------------------------------------------- look-up warps
+        const int lw = warp;
+        const int h = lane >> 4, l = lane & 15;
+        uint32_t colp[4];
+        make_colp<G>(colp, h, l);
+        unsigned job = 0;                     // table jobs (call, chunk) of this CTA, counted alike by every role
+        desc_begin(lw);
+        for (int c = c_begin; c < c_end; ++c) {
+            const ChainCall* d = desc_next(lw, c);
+            if (bid >= d->n_ctas) { __syncwarp(); continue; }
+            const ChainPart p = chain_part(d, bid);
+            const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
+            const uint8_t* seg_vp = d->tiles + ((size_t)p.kc0 * d->n_rb + p.rb0 + lw) * C::TILE_BYTES + lane * 16;
+            Item<Q, G> buf;
+            if (p.rb0 + lw < p.rb1) load_item<Q, G>(buf, seg_vp, seg_vp + (C::PLANE_BYTES - lane * 12), true);
+            for (int seg = 0; seg < p.nseg; ++seg, ++job) {
+                const int b = job & 1;
+                mbar_wait(bar_full(b), (job >> 1) & 1, spin_limit, status);
+                if (b == 0) chain_items<Q, G, 0>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, seg + 1 < p.nseg, seg_vp, tag, pf_ahead, lw, lane);
+                else chain_items<Q, G, 1>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, seg + 1 < p.nseg, seg_vp, tag, pf_ahead, lw, lane);
+                mbar_arrive(bar_free(b));     // this thread no longer reads buffer b
+                seg_vp += (size_t)d->n_rb * C::TILE_BYTES;
+            }
+            __syncwarp();                     // all lanes are done with descriptor c before its slot is refilled
+            if (d->n_kc == 1 && lane == 0 && !(d->flags & kCallTestNoSignal)) {
+                // no K split: this warp stored its rows of Y itself and reports them
+                __threadfence();
+                atomicAdd(done + c, 1u);
+            }
+        }
+    } else if (warp < kLookupWarps + kBuilderWarps) {
+        // ---------------------------------------------------------------- builder warps
+        const int bw = warp - kLookupWarps, bt = tid - kLookupWarps * 32;
+        unsigned job = 0;
+        for (int c = c_begin; c < c_end; ++c) {
+            const ChainCall* d = chain_desc(c);
+            // descriptor of the call after the next one (its slot was last read two calls ago)
+            if (c + 2 < c_end && bt < 8)
+                cp_async16(reinterpret_cast<uint8_t*>(chain_desc(c + 2)) + bt * 16, reinterpret_cast<const uint8_t*>(calls + (c + 2)) + bt * 16);
+            const bool work = bid < d->n_ctas;
+            ChainPart p = {0, 0, 0, 0, 0};
+            if (work) {
+                p = chain_part(d, bid);
+                // first items of the look-up warps: into L2 ahead of their register loads
+                for (int i = bt; i < kLookupWarps * pf_first; i += kBuilderThreads) {
+                    const int rb = p.rb0 + (i % kLookupWarps) + (i / kLookupWarps) * kLookupWarps;
+                    if (rb < p.rb1) prefetch_l2_bulk(d->tiles + ((size_t)p.kc0 * d->n_rb + rb) * C::TILE_BYTES, C::TILE_BYTES);
+                }
+            }
+            if (c + 1 < c_end && bt >= 32 && bt < 40) {
+                // activations of the next call's first chunk on this CTA: into L2 ahead of its table build
+                const ChainCall* dn = chain_desc(c + 1);
+                if (bid < dn->n_ctas) {
+                    const int k0 = (bid / dn->ranges) * dn->cpc * kChunkK + (bt - 32) * 64;
+                    if (k0 < dn->K) prefetch_l2_line(dn->X + k0);
+                }
+            }
+            if (bt == 0 && !sh->abort) {
+                bool ok = true;
+                // as-if-sequential order: every earlier call whose output this call reads or overwrites (or whose
+                // input it overwrites) is complete; calls of earlier launches are complete by stream order
+                for (int j = max(d->dep_first, c_begin); ok && j <= d->dep_last; ++j)
+                    ok = wait_reached(done + j, (epoch + 1u) * calls[j].done_target, spin_limit);
+                // the scratch region of this call was last used by call guard_call: its reductions must be over
+                if (ok && work && d->guard_call >= c_begin)
+                    ok = wait_reached(done + d->guard_call, (epoch + 1u) * calls[d->guard_call].done_target, spin_limit);
+                if (!ok) raise_abort(status);
+            }
+            if (bt < 8) cp_async_wait_all();
+            bar_builders();                   // the waits are over for all builder threads; descriptor c + 2 has landed
+            if (work) {
+                for (int seg = 0; seg < p.nseg; ++seg, ++job) {
+                    const int b = job & 1;
+                    if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);   // look-ups of job - 2 are over
+                    build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), d->X,
+                                       p.kc0 + seg, d->K, bw, lane);
+                    mbar_arrive(bar_full(b));
+                }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- finisher warps
+        // K-split reduction of every call this CTA works on, then the call's completion report
+        const int fw = warp - kLookupWarps - kBuilderWarps, ft = tid - (kLookupWarps + kBuilderWarps) * 32;
+        desc_begin(kLookupWarps + fw);
+        for (int c = c_begin; c < c_end; ++c) {
+            const ChainCall* d = desc_next(kLookupWarps + fw, c);
+            if (bid < d->n_ctas && d->n_kc > 1) {
+                const ChainPart p = chain_part(d, bid);
+                const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
+                chain_reduce(d, p, tag, spin_limit, status, ft);
+                bar_finishers();              // every row of this CTA is stored
+                if (ft == 0 && !(d->flags & kCallTestNoSignal)) {
+                    __threadfence();
+                    atomicAdd(done + c, 1u);
+                }
+            }
+            __syncwarp();
+        }
+        // the CTA that leaves the chain's last launch last opens the next epoch (completion counters and tags keep
+        // counting up across launches, so nothing has to be cleared); the finishers are the last of a CTA to be done
+        // with a call whose sums are split over K, the look-up warps with one that is not: both are waited for
+        bar_finishers();
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned t = atomicInc(&ctl->exit_ticket, gridDim.x - 1);
+        if (t == gridDim.x - 1 && last_run) ctl->epoch = epoch + 1u;
+    }
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct ChainLayout {
+    size_t done_off, calls_off, slots_off, region_bytes, total;
+};
+
+ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls) {
+    ChainLayout L;
+    size_t region = 0;
+    for (int i = 0; i < n_calls; ++i) {
+        const size_t n_rb = ((size_t)calls[i].N + kTileRows - 1) / kTileRows;
+        const size_t n_kc = ((size_t)calls[i].K + kChunkK - 1) / kChunkK;
+        const size_t b = n_kc > 1 ? n_kc * n_rb * kTileRows * sizeof(unsigned long long) : 0;
+        if (b > region) region = b;
+    }
+    L.region_bytes = round_up(region ? region : 256, 256);
+    L.done_off = 256;
+    L.calls_off = L.done_off + round_up((size_t)n_calls * sizeof(unsigned), 256);
+    L.slots_off = L.calls_off + round_up((size_t)n_calls * sizeof(ChainCall), 256);
+    L.total = L.slots_off + (size_t)kChainRegions * L.region_bytes;
+    return L;
+}
+
+int check_call(const elutq_gemv_call& c) {
+    if (!c.X || !c.packed || !c.Y) return ELUTQ_ERR_INVALID_ARG;
+    if (c.N <= 0 || c.K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    const unsigned known = ELUTQ_FLAG_OUT_F32 | ELUTQ_FLAG_ACCUMULATE | kCallTestNoSignal;
+    if (c.flags & ~(known | 0x3ffu)) return ELUTQ_ERR_INVALID_ARG;
+    if (c.flags & 0x3ffu & ~(ELUTQ_FLAG_OUT_F32 | ELUTQ_FLAG_ACCUMULATE)) return ELUTQ_ERR_UNSUPPORTED;
+    auto al = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    if (!al(c.X) || !al(c.packed) || !al(c.Y)) return ELUTQ_ERR_ALIGN;
+    return ELUTQ_OK;
+}
+
+template <int Q, int G>
+cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int last_run, unsigned wait_limit,
+                       int pf_first, int pf_ahead, int sms, cudaStream_t stream) {
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        e = cudaFuncSetAttribute(lut_chain_kernel<Q, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)sms);                   // one CTA per SM, all resident (cooperative launch)
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = kChainSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, lut_chain_kernel<Q, G>, ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead);
+    count_launch(1);
+    return e;
+}
+
+template <int Q>
+cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int last_run,
+                         unsigned wait_limit, int pf_first, int pf_ahead, int sms, cudaStream_t stream) {
+    switch (G) {
+        case 128: return launch_run<Q, 128>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
+        case 64: return launch_run<Q, 64>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
+        case 32: return launch_run<Q, 32>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+// Host-side copy of what elutq_chain_run needs of a plan (the runs of equal (q, G)), keyed by the plan's device
+// address; written by elutq_chain_plan.
+struct PlanRuns {
+    int n_calls = 0;
+    int n_runs = 0;
+    int begin[kMaxRuns + 1] = {};
+    int q[kMaxRuns] = {}, G[kMaxRuns] = {};
+    size_t calls_off = 0;
+};
+std::mutex g_plan_mu;
+std::map<const void*, PlanRuns> g_plans;
+
+}  // namespace
+}  // namespace elutq
+
+using namespace elutq;
+
+extern "C" {
+
+int elutq_chain_plan_bytes(const elutq_gemv_call* calls, int n_calls, size_t* bytes) {
+    if (!calls || !bytes || n_calls <= 0 || n_calls > ELUTQ_CHAIN_MAX_CALLS) return ELUTQ_ERR_INVALID_ARG;
+    for (int i = 0; i < n_calls; ++i) {
+        const int st = check_call(calls[i]);
+        if (st != ELUTQ_OK) return st;
+    }
+    *bytes = chain_layout(calls, n_calls).total;
+    return ELUTQ_OK;
+}
+
+int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size_t plan_bytes, void* stream) {
+    if (!plan) return ELUTQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    int st = elutq_chain_plan_bytes(calls, n_calls, &need);
+    if (st != ELUTQ_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(plan) & 255u) != 0) return ELUTQ_ERR_ALIGN;
+    if (plan_bytes < need) return ELUTQ_ERR_BUFFER_TOO_SMALL;
+    const ChainLayout L = chain_layout(calls, n_calls);
+    const int sms = device_sm_count();
+    uint8_t* base = reinterpret_cast<uint8_t*>(plan);
+
+    std::vector<uint8_t> host(L.slots_off, 0);
+    ChainCtl* ctl = reinterpret_cast<ChainCtl*>(host.data());
+    ctl->magic = kChainMagic;
+    ctl->n_calls = (unsigned)n_calls;
+    ctl->grid = (unsigned)sms;
+    ctl->done_off = L.done_off; ctl->calls_off = L.calls_off; ctl->slots_off = L.slots_off;
+    ctl->region_bytes = L.region_bytes; ctl->total_bytes = L.total;
+    ChainCall* dc = reinterpret_cast<ChainCall*>(host.data() + L.calls_off);
+    PlanRuns runs;
+    runs.n_calls = n_calls;
+    runs.calls_off = L.calls_off;
+    for (int i = 0; i < n_calls; ++i) {
+        const elutq_gemv_call& c = calls[i];
+        int q = 0, G = 0;
+        st = blob_meta(c.packed, c.N, c.K, &q, &G);       // reads the blob's header when the address is unknown
+        if (st != ELUTQ_OK) return st;
+        const Geo g = make_geo(q, G, c.N, c.K);
+        ChainCall& d = dc[i];
+        d.X = reinterpret_cast<const __half*>(c.X);
+        d.tiles = reinterpret_cast<const uint8_t*>(c.packed) + ELUTQ_HEADER_BYTES;
+        d.Y = c.Y;
+        d.slots = reinterpret_cast<unsigned long long*>(base + L.slots_off + (size_t)(i % kChainRegions) * L.region_bytes);
+        d.N = c.N; d.K = c.K; d.n_rb = g.n_rb; d.n_kc = g.n_kc;
+        d.q = q; d.G = G;
+        d.flags = c.flags & (ELUTQ_FLAG_OUT_F32 | ELUTQ_FLAG_ACCUMULATE | kCallTestNoSignal);
+        // as-if-sequential order: call i must follow every earlier call j whose output it reads (X_i on Y_j) or
+        // overwrites (Y_i on Y_j), or whose input it overwrites (Y_i on X_j)
+        d.dep_first = i; d.dep_last = -1;
+        for (int j = 0; j < i; ++j) {
+            const elutq_gemv_call& e = calls[j];
+            auto overlap = [](const void* a, size_t na, const void* b, size_t nb) {
+                const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b);
+                return pa < pb + nb && pb < pa + na;
+            };
+            const size_t xi = (size_t)c.K * 2, yi = (size_t)c.N * ((c.flags & ELUTQ_FLAG_OUT_F32) ? 4 : 2);
+            const size_t xj = (size_t)e.K * 2, yj = (size_t)e.N * ((e.flags & ELUTQ_FLAG_OUT_F32) ? 4 : 2);
+            if (overlap(c.X, xi, e.Y, yj) || overlap(c.Y, yi, e.Y, yj) || overlap(c.Y, yi, e.X, xj)) {
+                if (j < d.dep_first) d.dep_first = j;
+                d.dep_last = j;
+            }
+        }
+        int cpc = 1, R = 1;
+        plan_gemv_partition(g.n_rb, g.n_kc, sms, false, &cpc, &R);
+        d.cpc = cpc; d.ranges = R; d.rb_q = g.n_rb / R; d.rb_r = g.n_rb % R;
+        d.groups = (g.n_kc + cpc - 1) / cpc;
+        d.n_ctas = d.groups * R;
+        if (d.n_ctas > sms) return ELUTQ_ERR_UNSUPPORTED;
+        d.guard_call = i >= kChainRegions ? i - kChainRegions : -1;
+        d.done_target = (unsigned)(g.n_kc > 1 ? d.n_ctas : d.n_ctas * kLookupWarps);
+        if (runs.n_runs == 0 || runs.q[runs.n_runs - 1] != q || runs.G[runs.n_runs - 1] != G) {
+            if (runs.n_runs == kMaxRuns) return ELUTQ_ERR_UNSUPPORTED;
+            runs.begin[runs.n_runs] = i;
+            runs.q[runs.n_runs] = q;
+            runs.G[runs.n_runs] = G;
+            runs.n_runs += 1;
+        }
+    }
+    runs.begin[runs.n_runs] = n_calls;
+    cudaError_t e = cudaMemsetAsync(plan, 0, L.total, (cudaStream_t)stream);
+    if (e != cudaSuccess) return note_cuda_error((int)e);
+    // pageable source: the copy is staged by the runtime before the call returns
+    e = cudaMemcpyAsync(plan, host.data(), host.size(), cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    if (e != cudaSuccess) return note_cuda_error((int)e);
+    e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return note_cuda_error((int)e);
+    std::lock_guard<std::mutex> lk(g_plan_mu);
+    g_plans[plan] = runs;
+    return ELUTQ_OK;
+}
+
+int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefetch_first, int prefetch_ahead, void* stream) {
+    if (!plan || n_calls <= 0 || n_calls > ELUTQ_CHAIN_MAX_CALLS) return ELUTQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(plan) & 255u) != 0) return ELUTQ_ERR_ALIGN;
+    if (prefetch_first < 0 || prefetch_first > 8 || prefetch_ahead < 0 || prefetch_ahead > 1) return ELUTQ_ERR_INVALID_ARG;
+    PlanRuns runs;
+    {
+        std::lock_guard<std::mutex> lk(g_plan_mu);
+        auto it = g_plans.find(plan);
+        if (it == g_plans.end() || it->second.n_calls != n_calls) return ELUTQ_ERR_SHAPE;   // not planned by this process
+        runs = it->second;
+    }
+    ChainCtl* ctl = reinterpret_cast<ChainCtl*>(plan);
+    const ChainCall* calls = reinterpret_cast<const ChainCall*>(reinterpret_cast<uint8_t*>(plan) + runs.calls_off);
+    if (wait_limit == 0) wait_limit = 1u << 22;
+    const int sms = device_sm_count();
+    for (int r = 0; r < runs.n_runs; ++r) {
+        const int last = r + 1 == runs.n_runs;
+        cudaError_t e;
+        switch (runs.q[r]) {
+            case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
+            case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
+            case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
+            case 4: e = launch_run_q<4>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
+            default: e = cudaErrorInvalidValue; break;
+        }
+        if (e != cudaSuccess) return note_cuda_error((int)e);
+    }
+    return ELUTQ_OK;
+}
+
+int elutq_chain_run(void* plan, int n_calls, void* stream) {
+    return elutq_chain_run_opts(plan, n_calls, 0u, 2, 1, stream);
+}
+
+int elutq_chain_status(const void* plan, void* stream, int* status) {
+    if (!plan || !status) return ELUTQ_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return note_cuda_error((int)e);
+    ChainCtl h;
+    e = cudaMemcpy(&h, plan, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return note_cuda_error((int)e);
+    if (h.magic != kChainMagic) return ELUTQ_ERR_SHAPE;
+    *status = (int)h.status;
+    return ELUTQ_OK;
+}
+
+
+int elutq_chain_forget(const void* plan) {
+    if (!plan) return ELUTQ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_plan_mu);
+    g_plans.erase(plan);
+    return ELUTQ_OK;
+}
+
+}  // extern "C"

@@ -497,11 +497,11 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     b.items_q = (int)(total / grid);
     b.items_r = (int)(total % grid);
     b.active_warps = kWarps;
-    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.fused_reduce = 0; b.cpc = 1; b.cluster_reduce = 0;
+    b.ranges = 0; b.rb_q = 0; b.rb_r = 0; b.cpc = 1; b.cluster_reduce = 0;
     // Aligned partition when every (row batch, half chunk) segment can have its own CTAs: a CTA that straddles two
     // segments builds two table sets, which costs more than the slightly uneven ranges.
     const long long n_seg = (long long)n_mb * 2 * a.n_kc;
-    if (n_seg <= num_sms && debug_env("ELUTQ_DEBUG_FLAT") == 0) {
+    if (n_seg <= num_sms) {
         int R = (int)(num_sms / n_seg);
         if (R > a.n_rb) R = a.n_rb;
         if (R >= 1 && n_seg * R * 10 >= (long long)num_sms * 9) {      // only while it still uses >= 90 % of the SMs
@@ -521,7 +521,7 @@ int launch_mb(const GemmArgs& a, int num_sms, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = debug_env("ELUTQ_DEBUG_NO_PDL") > 0 ? 0 : 1;
+    cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, lut_gemm_kernel<Q, G, MB, TQ>, b);
     count_launch(1);
     if (e != cudaSuccess) return (int)e;
