@@ -234,7 +234,8 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  * decode step whose linears read separately produced activations streams without a pause, a chain in which
  * Y of one call is X of the next is run strictly in turn).
  *
- *   elutq_chain_plan_bytes  size of the plan buffer for a list (pure function, no CUDA call)
+ *   elutq_chain_plan_bytes  size of the plan buffer for a list on the current device (it depends on the SM count;
+ *                           nothing is launched)
  *   elutq_chain_plan        validates the list, reads q and G of every blob (elutq_describe's rules) and
  *                           writes the plan into `plan`: caller-owned DEVICE memory, 256-byte aligned, of
  *                           at least that size.  It holds the descriptors, the K-split scratch and the
@@ -247,10 +248,8 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  *                           nothing.  Runs of one plan must not overlap on the GPU.  Every CTA first
  *                           compares each blob's header with the plan; on a mismatch the launch ends at
  *                           once with status 0x7C0B and no tile is read.
- *   elutq_chain_run_opts    the same with explicit tuning values (test / measurement entry): the poll
- *                           limit of the hand-over waits (0 = default, 2^22), the number of items per warp
- *                           requested from L2 ahead of each call (0..8, default 2) and whether a rolling
- *                           L2 prefetch runs two items ahead of the register loads (0/1, default 1).
+ *   elutq_chain_run_opts    the same with an explicit poll limit for the hand-over waits (0 = default, 2^22);
+ *                           a test entry.
  *   elutq_chain_status      synchronises `stream` and reads the plan's status word: 0, or 0x7C05 after a
  *                           hand-over wait ran out (every wait is a bounded poll; the launch then finishes
  *                           without waiting any further and its results are undefined), or 0x7C0B.  After a
@@ -269,8 +268,7 @@ typedef struct elutq_gemv_call {
 int elutq_chain_plan_bytes(const elutq_gemv_call* calls, int n_calls, size_t* bytes);
 int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size_t plan_bytes, void* stream);
 int elutq_chain_run(void* plan, int n_calls, void* stream);
-int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefetch_first, int prefetch_ahead,
-                         void* stream);
+int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* stream);
 int elutq_chain_status(const void* plan, void* stream, int* status);
 /* The library keeps a small host-side note per planned buffer (which runs of equal (q, G) to launch);
  * elutq_chain_run returns ELUTQ_ERR_SHAPE for a buffer that this process has not planned.  Call this before

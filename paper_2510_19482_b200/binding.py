@@ -58,7 +58,7 @@ _SIGNATURES = {
     "elutq_chain_plan_bytes": (c_int, [ctypes.POINTER(GemvCall), c_int, ctypes.POINTER(c_size_t)]),
     "elutq_chain_plan": (c_int, [ctypes.POINTER(GemvCall), c_int, c_void_p, c_size_t, c_void_p]),
     "elutq_chain_run": (c_int, [c_void_p, c_int, c_void_p]),
-    "elutq_chain_run_opts": (c_int, [c_void_p, c_int, c_uint, c_int, c_int, c_void_p]),
+    "elutq_chain_run_opts": (c_int, [c_void_p, c_int, c_uint, c_void_p]),
     "elutq_chain_status": (c_int, [c_void_p, c_void_p, ctypes.POINTER(c_int)]),
     "elutq_chain_forget": (c_int, [c_void_p]),
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
@@ -241,10 +241,8 @@ def elutq_chain_run(plan, n_calls: int, stream=None) -> None:
     _check(lib().elutq_chain_run(_ptr(plan), n_calls, _stream(stream)), "elutq_chain_run")
 
 
-def elutq_chain_run_opts(plan, n_calls: int, wait_limit: int = 0, prefetch_first: int = 2, prefetch_ahead: int = 1,
-                         stream=None) -> None:
-    _check(lib().elutq_chain_run_opts(_ptr(plan), n_calls, wait_limit, prefetch_first, prefetch_ahead, _stream(stream)),
-           "elutq_chain_run_opts")
+def elutq_chain_run_opts(plan, n_calls: int, wait_limit: int = 0, stream=None) -> None:
+    _check(lib().elutq_chain_run_opts(_ptr(plan), n_calls, wait_limit, _stream(stream)), "elutq_chain_run_opts")
 
 
 def elutq_chain_status(plan, stream=None) -> int:

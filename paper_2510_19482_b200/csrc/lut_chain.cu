@@ -39,25 +39,27 @@ namespace {
 constexpr unsigned kChainMagic = 0x4E494843u;
 constexpr int kChainRegions = 3;              // scratch regions for the tagged partial sums, used round-robin
 constexpr int kDescSlots = 4;
-constexpr int kLookupWarps = 26;
+constexpr int kLookupWarps = 26;              // (22 or 18 look-up warps with 72 / 80 registers each measured slower)
 constexpr int kBuilderWarps = 4;
-constexpr int kFinisherWarps = kGemvWarps - kLookupWarps - kBuilderWarps;
+constexpr int kFinisherWarps = 2;
+constexpr int kChainThreads = (kLookupWarps + kBuilderWarps + kFinisherWarps) * 32;
 constexpr int kBuilderThreads = kBuilderWarps * 32;
 constexpr int kFinisherThreads = kFinisherWarps * 32;
 // shared memory: two table buffers, then per buffer 16 group sums, four mbarriers, flags, descriptor ring
 constexpr int kOffGsum = 2 * kTableBytes;
 constexpr int kOffBar = kOffGsum + 128;
 constexpr int kOffShared = kOffBar + 32;
+constexpr int kSlotBytes = 144;                           // descriptor (128) + this CTA's share of the call (16)
 constexpr int kOffDesc = kOffGsum + 256;                  // builders' descriptor ring
-constexpr int kOffWarpDesc = kOffDesc + kDescSlots * 128;   // look-up and finisher warps: two descriptor slots per warp
-constexpr int kChainSmem = kOffWarpDesc + (kLookupWarps + kFinisherWarps) * 2 * 128;
+constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // look-up and finisher warps: a descriptor ring per warp
+constexpr int kChainSmem = kOffWarpDesc + (kLookupWarps + kFinisherWarps) * kDescSlots * kSlotBytes;
 constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
 constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
 
 struct ChainCtl {                             // first 256 bytes of a plan
     unsigned magic, n_calls, status, epoch;
     unsigned exit_ticket, grid, reserved0, reserved1;
-    unsigned long long done_off, calls_off, slots_off, region_bytes, total_bytes;
+    unsigned long long done_off, calls_off, parts_off, slots_off, region_bytes, total_bytes;
 };
 
 struct ChainCall {                            // 128 bytes
@@ -93,9 +95,6 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ void prefetch_l2_bulk(const void* p, unsigned bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void prefetch_l2_line(const void* p) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
@@ -118,10 +117,12 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"((uint32_t)__cvta_generic_to_shared(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity) {
+// One bounded attempt: the thread is suspended by the hardware (it takes no issue slots from the other role's warps,
+// unlike a spinning test) until the phase completes or about a microsecond has passed.
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, unsigned parity) {
     unsigned ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity), "r"(1000u) : "memory");
     return ok != 0;
 }
 
@@ -133,11 +134,22 @@ struct ChainShared {
 extern __shared__ __align__(1024) uint8_t chain_smem[];
 
 __device__ __forceinline__ ChainShared* chain_shared() { return reinterpret_cast<ChainShared*>(chain_smem + kOffShared); }
-__device__ __forceinline__ ChainCall* chain_desc(int c) {
-    return reinterpret_cast<ChainCall*>(chain_smem + kOffDesc) + (c & (kDescSlots - 1));
+struct ChainSlot {                            // what a role keeps of a call in shared memory
+    ChainCall d;
+    int4 part;                                // this CTA's share: rb0, rb1, kc0, nseg | grp << 16
+};
+static_assert(sizeof(ChainSlot) == kSlotBytes, "slot size");
+__device__ __forceinline__ ChainSlot* chain_slot(int c) {
+    return reinterpret_cast<ChainSlot*>(chain_smem + kOffDesc) + (c & (kDescSlots - 1));
 }
-__device__ __forceinline__ ChainCall* warp_desc(int lw, int c) {
-    return reinterpret_cast<ChainCall*>(chain_smem + kOffWarpDesc) + lw * 2 + (c & 1);
+__device__ __forceinline__ ChainCall* chain_desc(int c) { return &chain_slot(c)->d; }
+__device__ __forceinline__ ChainSlot* warp_slot(int lw, int c) {
+    return reinterpret_cast<ChainSlot*>(chain_smem + kOffWarpDesc) + lw * kDescSlots + (c & (kDescSlots - 1));
+}
+// Copies descriptor c and this CTA's share of call c into a slot: nine 16-byte pieces, one per lane.
+__device__ __forceinline__ void slot_fetch(ChainSlot* dst, const ChainCall* calls, const int4* parts, int grid, int c, int piece) {
+    if (piece < 8) cp_async16(reinterpret_cast<uint8_t*>(dst) + piece * 16, reinterpret_cast<const uint8_t*>(calls + c) + piece * 16);
+    else if (piece == 8) cp_async16(&dst->part, parts + (size_t)c * grid + blockIdx.x);
 }
 __device__ __forceinline__ uint64_t* bar_full(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + b; }
 __device__ __forceinline__ uint64_t* bar_free(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + 2 + b; }
@@ -149,11 +161,11 @@ __device__ __forceinline__ void raise_abort(unsigned* status) {
         atomicExch(status, kStatusWaitExpired);
     }
 }
-// Bounded wait on a shared-memory barrier phase.
+// Bounded wait on a shared-memory barrier phase: at most limit / 64 suspended attempts of about a microsecond.
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, unsigned* status) {
     ChainShared* sh = chain_shared();
-    for (unsigned i = 0; !mbar_test(bar, parity); ++i) {
-        if (i >= limit || sh->abort) {
+    for (unsigned i = 0; !mbar_try(bar, parity); ++i) {
+        if (i >= (limit >> 6) + 16u || sh->abort) {
             raise_abort(status);
             return;
         }
@@ -183,14 +195,10 @@ __device__ __forceinline__ void chain_store(void* Y, unsigned flags, size_t idx,
 struct ChainPart {
     int rb0, rb1, kc0, nseg, grp;
 };
-__device__ __forceinline__ ChainPart chain_part(const ChainCall* d, int bid) {
+__device__ __forceinline__ ChainPart chain_part(const ChainSlot* s) {
     ChainPart p;
-    p.grp = bid / d->ranges;
-    const int range = bid - p.grp * d->ranges;
-    p.rb0 = range * d->rb_q + min(range, d->rb_r);
-    p.rb1 = p.rb0 + d->rb_q + (range < d->rb_r ? 1 : 0);
-    p.kc0 = p.grp * d->cpc;
-    p.nseg = min(d->cpc, d->n_kc - p.kc0);
+    p.rb0 = s->part.x; p.rb1 = s->part.y; p.kc0 = s->part.z;
+    p.nseg = s->part.w & 0xffff; p.grp = s->part.w >> 16;
     return p;
 }
 
@@ -235,15 +243,9 @@ __device__ __noinline__ void chain_reduce(const ChainCall* d, const ChainPart p,
     }
 }
 
-// Fused tables of chunk kc (and its group sums) built by the builder warps: lane -> column pair (2*lane,
-// 2*lane+1) as in build_tables; builder warp bw takes the (high nibble, low-nibble half) combinations
-// vw = bw, bw + 4, ... of the 32 that a full CTA would spread over its warps.
-template <int G>
-__device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const __half* __restrict__ X, int kc, int K,
-                                                int bw, int lane) {
-    constexpr int W = G / 8;
+// The lane's 16 activations of chunk kc (two byte-columns), as (x_i of column 2*lane, x_i of column 2*lane+1).
+__device__ __forceinline__ void load_x_pairs(float2 (&x)[8], const __half* __restrict__ X, int kc, int K, int lane) {
     const int k0 = kc * kChunkK + lane * 16;
-    float2 x[8];
     if (k0 < K) {
         const uint4 r0 = __ldcg(reinterpret_cast<const uint4*>(X + k0));      // past the incoherent L1: X may have
         const uint4 r1 = __ldcg(reinterpret_cast<const uint4*>(X + k0 + 8));  // been written during this launch
@@ -259,6 +261,13 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 #pragma unroll
         for (int i = 0; i < 8; ++i) x[i] = make_float2(0.f, 0.f);
     }
+}
+// Fused tables of a chunk (and its group sums) built by the builder warps from the activations x: lane -> column
+// pair (2*lane, 2*lane+1) as in build_tables; builder warp bw takes the (high nibble, low-nibble half) combinations
+// vw = bw, bw + 4, ... of the 32 that a full CTA would spread over its warps.
+template <int G>
+__device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const float2 (&x)[8], int bw, int lane) {
+    constexpr int W = G / 8;
 #pragma unroll
     for (int lh = 0; lh < 2; ++lh) {
         float2 A[8];
@@ -292,11 +301,12 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 }
 
 // Items of one chunk (kc) of call d on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of
-// the chunk on entry and its first item of the next chunk (when there is one) on exit.
+// the chunk on entry and, on exit, the item at after_vp (its first item of the CTA's next chunk or of the next
+// call; nullptr: none).
 template <int Q, int G, int B>
 __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const ChainCall* d, const int rb0,
-                                            const int rb1, const int kc, const bool more_segs, const uint8_t* seg_vp,
-                                            const unsigned tag, const int pf_ahead, const int lw, const int lane) {
+                                            const int rb1, const int kc, const uint8_t* after_vp, const uint8_t* seg_vp,
+                                            const unsigned tag, const int lw, const int lane) {
     using C = Cfg<Q, G>;
     const uint8_t* const tab = chain_smem + B * kTableBytes;
     const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
@@ -304,18 +314,15 @@ __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&co
     float S[C::GL];
     load_group_sums<G>(S, gsum, h, l, true);
     const int n_rb = d->n_rb;
-    const uint8_t* next_seg_vp = seg_vp + (size_t)n_rb * C::TILE_BYTES;
     const uint8_t* vp = seg_vp;
     unsigned long long* out = d->slots + (size_t)kc * ((size_t)n_rb * kTileRows) + l;
     for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
-        // next item of this warp: the same chunk, else its first item of the CTA's next chunk
+        // next item of this warp: the same chunk, else the one the caller names
         const bool in_seg = rb + kLookupWarps < rb1;
-        const uint8_t* nvp = in_seg ? vp + kLookupWarps * C::TILE_BYTES : next_seg_vp;
+        const uint8_t* nvp = in_seg ? vp + kLookupWarps * C::TILE_BYTES : after_vp;
         const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
-        if (pf_ahead > 0 && lane == 0 && rb + 2 * kLookupWarps < rb1)   // rolling L2 prefetch, one item beyond the register loads
-            prefetch_l2_bulk(vp + 2 * kLookupWarps * C::TILE_BYTES, C::TILE_BYTES);
         float y;
-        if (in_seg || more_segs) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
+        if (in_seg || after_vp != nullptr) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
         else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
         if (h == 0) {
             if (d->n_kc == 1) {
@@ -328,30 +335,128 @@ __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&co
     }
 }
 
+// What the roles of a launch share.
+struct ChainCtx {
+    const ChainCall* calls;
+    const int4* parts;
+    unsigned* done;
+    unsigned* status;
+    int grid, n_calls, c_begin, c_end;
+    unsigned epoch, spin_limit;
+};
+
+// Per-warp descriptor copies for the warps that run on their own (look-up and finisher warps): the copies of
+// calls c + 1 and c + 2 are on their way or there while call c is worked on.
+__device__ __forceinline__ void desc_fetch(const ChainCtx& x, int slot_warp, int c, int lane) {
+    if (lane < 9 && c < x.c_end) slot_fetch(warp_slot(slot_warp, c), x.calls, x.parts, x.grid, c, lane);
+}
+__device__ __forceinline__ void desc_begin(const ChainCtx& x, int slot_warp, int lane) {
+    desc_fetch(x, slot_warp, x.c_begin, lane);
+    desc_fetch(x, slot_warp, x.c_begin + 1, lane);
+    if (lane < 9) cp_async_wait_all();
+    __syncwarp();
+}
+// descriptor of call c for this warp; call c + 1 has landed too, call c + 2 is requested
+__device__ __forceinline__ const ChainSlot* desc_next(const ChainCtx& x, int slot_warp, int c, int lane) {
+    if (lane < 9) cp_async_wait_all();            // c + 1 (requested one call ago)
+    __syncwarp();                                 // ... and nobody still reads the slot of call c - 2
+    desc_fetch(x, slot_warp, c + 2, lane);
+    if (lane < 9) asm volatile("cp.async.commit_group;" ::: "memory");
+    return warp_slot(slot_warp, c);
+}
+
+// Look-up role of one warp over the calls of a launch.  (A launch covers calls of one (q, G): a variant that switched
+// between per-q instances of this function inside one kernel was measured three times slower, whether the instances
+// were inlined or called.)
+template <int Q, int G>
+__device__ __forceinline__ void lookup_calls(const ChainCtx& x) {
+    using C = Cfg<Q, G>;
+    const int lane = threadIdx.x & 31, lw = threadIdx.x >> 5, bid = blockIdx.x;
+    const int h = lane >> 4, l = lane & 15;
+    uint32_t colp[4];
+    make_colp<G>(colp, h, l);
+    unsigned job = 0;                         // table jobs (call, chunk) of this CTA, counted alike by every role
+    Item<Q, G> buf;
+    bool carried = false;                     // buf already holds this warp's first item of the call
+    desc_begin(x, lw, lane);
+    for (int c = x.c_begin; c < x.c_end; ++c) {
+        const ChainSlot* sl = desc_next(x, lw, c, lane);
+        const ChainCall* d = &sl->d;
+        if (bid >= d->n_ctas) continue;
+        const ChainPart p = chain_part(sl);
+        const unsigned tag = x.epoch * (unsigned)x.n_calls + (unsigned)c + 1u;
+        const uint8_t* seg_vp = d->tiles + ((size_t)p.kc0 * d->n_rb + p.rb0 + lw) * C::TILE_BYTES + lane * 16;
+        const bool items = p.rb0 + lw < p.rb1;
+        if (items && !carried) load_item<Q, G>(buf, seg_vp, seg_vp + (C::PLANE_BYTES - lane * 12), true);
+        carried = false;
+        // what follows this warp's last item of the call: its first item of the next call, when the CTA and the
+        // warp have work there
+        const uint8_t* next_call_vp = nullptr;
+        if (items && c + 1 < x.c_end) {
+            const ChainSlot* sn = warp_slot(lw, c + 1);
+            const ChainCall* dn = &sn->d;
+            if (bid < dn->n_ctas) {
+                const ChainPart pn = chain_part(sn);
+                if (pn.rb0 + lw < pn.rb1) {
+                    next_call_vp = dn->tiles + ((size_t)pn.kc0 * dn->n_rb + pn.rb0 + lw) * C::TILE_BYTES + lane * 16;
+                    carried = true;
+                }
+            }
+        }
+        for (int seg = 0; seg < p.nseg; ++seg, ++job) {
+            const int b = job & 1;
+            const uint8_t* after_vp = seg + 1 < p.nseg ? seg_vp + (size_t)d->n_rb * C::TILE_BYTES : next_call_vp;
+            mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
+            if (b == 0) chain_items<Q, G, 0>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
+            else chain_items<Q, G, 1>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
+            mbar_arrive(bar_free(b));         // this thread no longer reads buffer b
+            seg_vp += (size_t)d->n_rb * C::TILE_BYTES;
+        }
+        if (d->n_kc == 1) {
+            __syncwarp();
+            if (lane == 0 && !(d->flags & kCallTestNoSignal)) {
+                // no K split: this warp stored its rows of Y itself and reports them
+                __threadfence();
+                atomicAdd(x.done + c, 1u);
+            }
+        }
+    }
+}
+
 // Calls [c_begin, c_end) of the plan, all with the kernel's (Q, G).
 template <int Q, int G>
-__global__ void __launch_bounds__(kGemvThreads, 1)
+__global__ void __launch_bounds__(kChainThreads, 1)
 lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const int c_begin, const int c_end,
-                 const int last_run, const unsigned spin_limit, const int pf_first, const int pf_ahead) {
-    using C = Cfg<Q, G>;
+                 const int first_run, const int last_run, const unsigned spin_limit) {
     uint8_t* const smem = chain_smem;
     ChainShared* sh = chain_shared();
     unsigned* done = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(ctl) + ctl->done_off);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bid = blockIdx.x;
 
+    // The launches of a chain follow one another by programmatic dependent launch: a CTA of the next launch starts
+    // on an SM as soon as this launch's CTA there has left (every launch fills the device, one CTA per SM).  Only the
+    // chain's first launch waits for whatever precedes the chain in the stream (and for the previous run of this plan,
+    // which advances the epoch at its very end); it releases its successor after that wait, so the guarantee carries
+    // over.  Data dependencies between calls of different launches go through the completion counters like those
+    // inside a launch.
+    if (first_run) grid_dependency_wait();
+    grid_launch_dependents();
+
     // Before any tile is read: the plan is the one the host launched, and every blob of this run still carries
     // the header it was planned with.
     int bad = (ctl->magic != kChainMagic || ctl->n_calls != (unsigned)n_calls) ? 1 : 0;
     if (!bad) {
-        for (int c = c_begin + tid; c < c_end; c += kGemvThreads) {
+        for (int c = c_begin + tid; c < c_end; c += kChainThreads) {
             const ChainCall* d = calls + c;
             if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) bad = 1;
         }
     }
-    if (tid < 8 * min(c_end - c_begin, 2)) {
-        const int c = c_begin + (tid >> 3);
-        cp_async16(reinterpret_cast<uint8_t*>(chain_desc(c)) + (tid & 7) * 16, reinterpret_cast<const uint8_t*>(calls + c) + (tid & 7) * 16);
+    const int4* parts = reinterpret_cast<const int4*>(reinterpret_cast<const uint8_t*>(ctl) + ctl->parts_off);
+    const int grid = (int)gridDim.x;
+    if (tid < 16 * min(c_end - c_begin, 3)) {
+        const int c = c_begin + (tid >> 4);
+        slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
     }
     if (tid == 0) {
         sh->abort = 0;
@@ -370,115 +475,78 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
     const unsigned epoch = sh->epoch;
     unsigned* const status = &ctl->status;
 
-    // Per-warp descriptor copies for the warps that run on their own (look-up and finisher warps): the copy of
-    // call c + 1 is fetched while call c is worked on.
-    auto desc_begin = [&](int slot_warp) {
-        if (lane < 8) cp_async16(reinterpret_cast<uint8_t*>(warp_desc(slot_warp, c_begin)) + lane * 16,
-                                 reinterpret_cast<const uint8_t*>(calls + c_begin) + lane * 16);
-    };
-    auto desc_next = [&](int slot_warp, int c) -> const ChainCall* {
-        if (lane < 8) {
-            cp_async_wait_all();
-            if (c + 1 < c_end) {
-                cp_async16(reinterpret_cast<uint8_t*>(warp_desc(slot_warp, c + 1)) + lane * 16,
-                           reinterpret_cast<const uint8_t*>(calls + (c + 1)) + lane * 16);
-                asm volatile("cp.async.commit_group;" ::: "memory");
-            }
-        }
-        __syncwarp();
-        return warp_desc(slot_warp, c);
-    };
+    ChainCtx x;
+    x.calls = calls; x.parts = parts; x.done = done; x.status = status;
+    x.grid = grid; x.n_calls = n_calls; x.c_begin = c_begin; x.c_end = c_end;
+    x.epoch = epoch; x.spin_limit = spin_limit;
 
     if (warp < kLookupWarps) {
         // ---------------------------------------------------------------- look-up warps
-        const int lw = warp;
-        const int h = lane >> 4, l = lane & 15;
-        uint32_t colp[4];
-        make_colp<G>(colp, h, l);
-        unsigned job = 0;                     // table jobs (call, chunk) of this CTA, counted alike by every role
-        desc_begin(lw);
-        for (int c = c_begin; c < c_end; ++c) {
-            const ChainCall* d = desc_next(lw, c);
-            if (bid >= d->n_ctas) { __syncwarp(); continue; }
-            const ChainPart p = chain_part(d, bid);
-            const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
-            const uint8_t* seg_vp = d->tiles + ((size_t)p.kc0 * d->n_rb + p.rb0 + lw) * C::TILE_BYTES + lane * 16;
-            Item<Q, G> buf;
-            if (p.rb0 + lw < p.rb1) load_item<Q, G>(buf, seg_vp, seg_vp + (C::PLANE_BYTES - lane * 12), true);
-            for (int seg = 0; seg < p.nseg; ++seg, ++job) {
-                const int b = job & 1;
-                mbar_wait(bar_full(b), (job >> 1) & 1, spin_limit, status);
-                if (b == 0) chain_items<Q, G, 0>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, seg + 1 < p.nseg, seg_vp, tag, pf_ahead, lw, lane);
-                else chain_items<Q, G, 1>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, seg + 1 < p.nseg, seg_vp, tag, pf_ahead, lw, lane);
-                mbar_arrive(bar_free(b));     // this thread no longer reads buffer b
-                seg_vp += (size_t)d->n_rb * C::TILE_BYTES;
-            }
-            __syncwarp();                     // all lanes are done with descriptor c before its slot is refilled
-            if (d->n_kc == 1 && lane == 0 && !(d->flags & kCallTestNoSignal)) {
-                // no K split: this warp stored its rows of Y itself and reports them
-                __threadfence();
-                atomicAdd(done + c, 1u);
-            }
-        }
+        lookup_calls<Q, G>(x);
     } else if (warp < kLookupWarps + kBuilderWarps) {
         // ---------------------------------------------------------------- builder warps
         const int bw = warp - kLookupWarps, bt = tid - kLookupWarps * 32;
         unsigned job = 0;
         for (int c = c_begin; c < c_end; ++c) {
             const ChainCall* d = chain_desc(c);
-            // descriptor of the call after the next one (its slot was last read two calls ago)
-            if (c + 2 < c_end && bt < 8)
-                cp_async16(reinterpret_cast<uint8_t*>(chain_desc(c + 2)) + bt * 16, reinterpret_cast<const uint8_t*>(calls + (c + 2)) + bt * 16);
+            // descriptor three calls ahead (its slot was last read one call ago); it is waited for at the end of this
+            // iteration and published by the barrier of the next one
+            if (c + 3 < c_end && bt < 9) slot_fetch(chain_slot(c + 3), calls, parts, grid, c + 3, bt);
             const bool work = bid < d->n_ctas;
             ChainPart p = {0, 0, 0, 0, 0};
             if (work) {
-                p = chain_part(d, bid);
-                // first items of the look-up warps: into L2 ahead of their register loads
-                for (int i = bt; i < kLookupWarps * pf_first; i += kBuilderThreads) {
-                    const int rb = p.rb0 + (i % kLookupWarps) + (i / kLookupWarps) * kLookupWarps;
-                    if (rb < p.rb1) prefetch_l2_bulk(d->tiles + ((size_t)p.kc0 * d->n_rb + rb) * C::TILE_BYTES, C::TILE_BYTES);
-                }
+                p = chain_part(chain_slot(c));
             }
             if (c + 1 < c_end && bt >= 32 && bt < 40) {
                 // activations of the next call's first chunk on this CTA: into L2 ahead of its table build
                 const ChainCall* dn = chain_desc(c + 1);
                 if (bid < dn->n_ctas) {
-                    const int k0 = (bid / dn->ranges) * dn->cpc * kChunkK + (bt - 32) * 64;
+                    const int k0 = chain_slot(c + 1)->part.z * kChunkK + (bt - 32) * 64;
                     if (k0 < dn->K) prefetch_l2_line(dn->X + k0);
                 }
             }
-            if (bt == 0 && !sh->abort) {
-                bool ok = true;
+            if (d->dep_first <= d->dep_last) {
                 // as-if-sequential order: every earlier call whose output this call reads or overwrites (or whose
-                // input it overwrites) is complete; calls of earlier launches are complete by stream order
-                for (int j = max(d->dep_first, c_begin); ok && j <= d->dep_last; ++j)
-                    ok = wait_reached(done + j, (epoch + 1u) * calls[j].done_target, spin_limit);
-                // the scratch region of this call was last used by call guard_call: its reductions must be over
-                if (ok && work && d->guard_call >= c_begin)
-                    ok = wait_reached(done + d->guard_call, (epoch + 1u) * calls[d->guard_call].done_target, spin_limit);
-                if (!ok) raise_abort(status);
+                // input it overwrites) is complete
+                if (bt == 0 && !sh->abort) {
+                    bool ok = true;
+                    for (int j = d->dep_first; ok && j <= d->dep_last; ++j)
+                        ok = wait_reached(done + j, (epoch + 1u) * calls[j].done_target, spin_limit);
+                    if (!ok) raise_abort(status);
+                }
+                bar_builders();
             }
-            if (bt < 8) cp_async_wait_all();
-            bar_builders();                   // the waits are over for all builder threads; descriptor c + 2 has landed
             if (work) {
                 for (int seg = 0; seg < p.nseg; ++seg, ++job) {
                     const int b = job & 1;
+                    float2 xv[8];             // requested before the wait for the buffer: the load latency overlaps it
+                    load_x_pairs(xv, d->X, p.kc0 + seg, d->K, lane);
                     if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);   // look-ups of job - 2 are over
-                    build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), d->X,
-                                       p.kc0 + seg, d->K, bw, lane);
+                    build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), xv, bw, lane);
+                    if (seg == 0 && d->guard_call >= 0) {
+                        // the scratch region of this call was last used by call guard_call: its reductions must be over
+                        // before the look-up warps store into it (they start when the tables are handed over)
+                        if (bt == 0 && !sh->abort &&
+                            !wait_reached(done + d->guard_call, (epoch + 1u) * calls[d->guard_call].done_target, spin_limit))
+                            raise_abort(status);
+                        bar_builders();
+                    }
                     mbar_arrive(bar_full(b));
                 }
             }
+            if (bt < 9) cp_async_wait_all();
+            bar_builders();                   // descriptor c + 3 has landed for every builder thread
         }
     } else {
         // ---------------------------------------------------------------- finisher warps
         // K-split reduction of every call this CTA works on, then the call's completion report
         const int fw = warp - kLookupWarps - kBuilderWarps, ft = tid - (kLookupWarps + kBuilderWarps) * 32;
-        desc_begin(kLookupWarps + fw);
+        desc_begin(x, kLookupWarps + fw, lane);
         for (int c = c_begin; c < c_end; ++c) {
-            const ChainCall* d = desc_next(kLookupWarps + fw, c);
+            const ChainSlot* sl = desc_next(x, kLookupWarps + fw, c, lane);
+            const ChainCall* d = &sl->d;
             if (bid < d->n_ctas && d->n_kc > 1) {
-                const ChainPart p = chain_part(d, bid);
+                const ChainPart p = chain_part(sl);
                 const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
                 chain_reduce(d, p, tag, spin_limit, status, ft);
                 bar_finishers();              // every row of this CTA is stored
@@ -495,20 +563,21 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
         bar_finishers();
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0 && last_run) {
+        // (when every CTA of the chain's last launch has started, every CTA of the launches before it has left)
         __threadfence();
         const unsigned t = atomicInc(&ctl->exit_ticket, gridDim.x - 1);
-        if (t == gridDim.x - 1 && last_run) ctl->epoch = epoch + 1u;
+        if (t == gridDim.x - 1) ctl->epoch = epoch + 1u;
     }
 }
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct ChainLayout {
-    size_t done_off, calls_off, slots_off, region_bytes, total;
+    size_t done_off, calls_off, parts_off, slots_off, region_bytes, total;
 };
 
-ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls) {
+ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls, int sms) {
     ChainLayout L;
     size_t region = 0;
     for (int i = 0; i < n_calls; ++i) {
@@ -520,7 +589,8 @@ ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls) {
     L.region_bytes = round_up(region ? region : 256, 256);
     L.done_off = 256;
     L.calls_off = L.done_off + round_up((size_t)n_calls * sizeof(unsigned), 256);
-    L.slots_off = L.calls_off + round_up((size_t)n_calls * sizeof(ChainCall), 256);
+    L.parts_off = L.calls_off + round_up((size_t)n_calls * sizeof(ChainCall), 256);
+    L.slots_off = L.parts_off + round_up((size_t)n_calls * sms * sizeof(int4), 256);
     L.total = L.slots_off + (size_t)kChainRegions * L.region_bytes;
     return L;
 }
@@ -537,8 +607,8 @@ int check_call(const elutq_gemv_call& c) {
 }
 
 template <int Q, int G>
-cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int last_run, unsigned wait_limit,
-                       int pf_first, int pf_ahead, int sms, cudaStream_t stream) {
+cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int first_run, int last_run,
+                       unsigned wait_limit, int sms, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -550,26 +620,33 @@ cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)sms);                   // one CTA per SM, all resident (cooperative launch)
-    cfg.blockDim = dim3(kGemvThreads);
+    cfg.blockDim = dim3(kChainThreads);
     cfg.dynamicSmemBytes = kChainSmem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    // The chain's first launch is cooperative (its CTAs wait on one another: the runtime guarantees that all are
+    // resident).  Later launches follow by programmatic dependent launch instead, which lets their CTAs move in as
+    // the predecessor's leave (the two attributes together were measured to serialise the launches: 109 against 98 us
+    // on the twelve calls of three bit-widths); they fill the device in the same way - one CTA per SM, as many CTAs
+    // as SMs - so all of them become resident as soon as the predecessor has drained, and every wait is bounded.
+    cfg.attrs = first_run ? attr : attr + 1;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, lut_chain_kernel<Q, G>, ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead);
+    e = cudaLaunchKernelEx(&cfg, lut_chain_kernel<Q, G>, ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit);
     count_launch(1);
     return e;
 }
 
 template <int Q>
-cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int last_run,
-                         unsigned wait_limit, int pf_first, int pf_ahead, int sms, cudaStream_t stream) {
+cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int first_run, int last_run,
+                         unsigned wait_limit, int sms, cudaStream_t stream) {
     switch (G) {
-        case 128: return launch_run<Q, 128>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
-        case 64: return launch_run<Q, 64>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
-        case 32: return launch_run<Q, 32>(ctl, calls, n_calls, c0, c1, last_run, wait_limit, pf_first, pf_ahead, sms, stream);
+        case 128: return launch_run<Q, 128>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
+        case 64: return launch_run<Q, 64>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
+        case 32: return launch_run<Q, 32>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -599,7 +676,7 @@ int elutq_chain_plan_bytes(const elutq_gemv_call* calls, int n_calls, size_t* by
         const int st = check_call(calls[i]);
         if (st != ELUTQ_OK) return st;
     }
-    *bytes = chain_layout(calls, n_calls).total;
+    *bytes = chain_layout(calls, n_calls, device_sm_count()).total;
     return ELUTQ_OK;
 }
 
@@ -610,8 +687,8 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
     if (st != ELUTQ_OK) return st;
     if ((reinterpret_cast<uintptr_t>(plan) & 255u) != 0) return ELUTQ_ERR_ALIGN;
     if (plan_bytes < need) return ELUTQ_ERR_BUFFER_TOO_SMALL;
-    const ChainLayout L = chain_layout(calls, n_calls);
     const int sms = device_sm_count();
+    const ChainLayout L = chain_layout(calls, n_calls, sms);
     uint8_t* base = reinterpret_cast<uint8_t*>(plan);
 
     std::vector<uint8_t> host(L.slots_off, 0);
@@ -619,7 +696,7 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
     ctl->magic = kChainMagic;
     ctl->n_calls = (unsigned)n_calls;
     ctl->grid = (unsigned)sms;
-    ctl->done_off = L.done_off; ctl->calls_off = L.calls_off; ctl->slots_off = L.slots_off;
+    ctl->done_off = L.done_off; ctl->calls_off = L.calls_off; ctl->parts_off = L.parts_off; ctl->slots_off = L.slots_off;
     ctl->region_bytes = L.region_bytes; ctl->total_bytes = L.total;
     ChainCall* dc = reinterpret_cast<ChainCall*>(host.data() + L.calls_off);
     PlanRuns runs;
@@ -661,6 +738,20 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
         d.groups = (g.n_kc + cpc - 1) / cpc;
         d.n_ctas = d.groups * R;
         if (d.n_ctas > sms) return ELUTQ_ERR_UNSUPPORTED;
+        // every CTA's share of the call: row-block range, first chunk, chunks, chunk group
+        int4* pt = reinterpret_cast<int4*>(host.data() + L.parts_off) + (size_t)i * sms;
+        for (int b = 0; b < sms; ++b) {
+            int4 v = make_int4(0, 0, 0, 0);
+            if (b < d.n_ctas) {
+                const int grp = b / R, range = b - grp * R;
+                v.x = range * d.rb_q + (range < d.rb_r ? range : d.rb_r);
+                v.y = v.x + d.rb_q + (range < d.rb_r ? 1 : 0);
+                v.z = grp * cpc;
+                const int nseg = (cpc < g.n_kc - v.z) ? cpc : g.n_kc - v.z;
+                v.w = nseg | (grp << 16);
+            }
+            pt[b] = v;
+        }
         d.guard_call = i >= kChainRegions ? i - kChainRegions : -1;
         d.done_target = (unsigned)(g.n_kc > 1 ? d.n_ctas : d.n_ctas * kLookupWarps);
         if (runs.n_runs == 0 || runs.q[runs.n_runs - 1] != q || runs.G[runs.n_runs - 1] != G) {
@@ -684,10 +775,9 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
     return ELUTQ_OK;
 }
 
-int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefetch_first, int prefetch_ahead, void* stream) {
+int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* stream) {
     if (!plan || n_calls <= 0 || n_calls > ELUTQ_CHAIN_MAX_CALLS) return ELUTQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(plan) & 255u) != 0) return ELUTQ_ERR_ALIGN;
-    if (prefetch_first < 0 || prefetch_first > 8 || prefetch_ahead < 0 || prefetch_ahead > 1) return ELUTQ_ERR_INVALID_ARG;
     PlanRuns runs;
     {
         std::lock_guard<std::mutex> lk(g_plan_mu);
@@ -703,10 +793,10 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefe
         const int last = r + 1 == runs.n_runs;
         cudaError_t e;
         switch (runs.q[r]) {
-            case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
-            case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
-            case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
-            case 4: e = launch_run_q<4>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], last, wait_limit, prefetch_first, prefetch_ahead, sms, (cudaStream_t)stream); break;
+            case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 4: e = launch_run_q<4>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
             default: e = cudaErrorInvalidValue; break;
         }
         if (e != cudaSuccess) return note_cuda_error((int)e);
@@ -715,7 +805,7 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, int prefe
 }
 
 int elutq_chain_run(void* plan, int n_calls, void* stream) {
-    return elutq_chain_run_opts(plan, n_calls, 0u, 2, 1, stream);
+    return elutq_chain_run_opts(plan, n_calls, 0u, stream);
 }
 
 int elutq_chain_status(const void* plan, void* stream, int* status) {
