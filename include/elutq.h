@@ -125,19 +125,28 @@ int elutq_unpack(const void* packed, int N, int K, uint8_t* planes, void* scales
                  void* offsets, void* stream);
 
 /*
- * Reads q and G of a blob.  Blobs produced by elutq_pack in this process are
- * known to the library; for any other device address the 128-byte header is
- * copied to the host once (a synchronous cudaMemcpy) and remembered.
- * Any of q, G may be NULL.  ELUTQ_ERR_SHAPE if the header is not a valid blob
- * for (N, K).
+ * Reads q and G of the blob that is at `packed` now: the 128-byte header is copied
+ * to the host (a synchronous cudaMemcpy - not during stream capture) and what the
+ * library remembers about the address is refreshed.  Any of q, G may be NULL.
+ * ELUTQ_ERR_SHAPE if the header is not a valid blob for (N, K).
+ *
+ * The GEMM entry points remember (q, G, N, K) per device address - from elutq_pack,
+ * from this call, or from a header read on first use - so that a call costs no
+ * copy.  A remembered description can go stale (the buffer was freed and its
+ * address now holds another blob that arrived by a plain copy).  That is caught on
+ * the device: every kernel that reads tiles first compares the blob's header with
+ * the (q, G, N, K) it was launched for and, on a mismatch, raises the device status
+ * ELUTQ_DEVICE_BLOB_MISMATCH and returns without reading a tile or writing Y.
+ * Call elutq_describe (or elutq_forget) after replacing a blob in place.
  */
 int elutq_describe(const void* packed, int N, int K, int* q, int* G);
 
-/* Forget what the library remembers about `packed`.  The library keys what it
- * knows (q, G, N, K) by device address and refreshes it on elutq_pack and when
- * (N, K) disagree; call this before freeing a blob if its address may later hold
- * a blob of the same (N, K) but different q or G that arrives by a plain copy. */
+/* Forget what the library remembers about `packed` (the next use reads the header). */
 int elutq_forget(const void* packed);
+
+/* Device status words (elutq_device_status, elutq_chain_status). */
+#define ELUTQ_DEVICE_WAIT_EXPIRED  0x7C05 /* a bounded device-side wait ran out                        */
+#define ELUTQ_DEVICE_BLOB_MISMATCH 0x7C0B /* a blob's header did not match what the kernel was given   */
 
 /*
  * Scratch memory the GEMM needs for (M,N,K): a small reserved control area and the
@@ -156,13 +165,34 @@ int elutq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * Y[M,N] = X[M,K] * W_hat^T with scales and offsets applied (Eq. 3 under the
  * bit-serial LUT procedure of Appendix B), fp32 tables and accumulation, one
  * round-to-nearest-even conversion to fp16 at the end.
- *   X, Y, packed: device.  Scratch comes from a library-owned per-(device,stream)
- *   buffer that is allocated with cudaMalloc on the first call that needs it (or
- *   needs a larger one): make one warm-up call before capturing into a CUDA graph.
+ *   X, Y, packed: device.  `packed` must be complete when the call is enqueued:
+ *   the kernels start reading it before they wait for the work that precedes
+ *   them on the stream (weights do not depend on the previous kernel; X, Y and the
+ *   scratch do).  After elutq_pack on the same stream that holds - pack kernels
+ *   run to completion before a dependent launch starts - but a producer of
+ *   `packed` that triggers programmatic dependent launches early must be
+ *   synchronised with first.
+ *   Scratch comes from library-owned buffers per (device, stream), allocated with
+ *   cudaMalloc on the first call that needs them or needs larger ones.  A buffer
+ *   that has to grow is replaced, never freed: the old one stays allocated until
+ *   elutq_release_scratch, because a CUDA graph captured earlier still carries its
+ *   address.  While `stream` is being captured nothing is allocated: a call that
+ *   would need more scratch than the stream has returns
+ *   ELUTQ_ERR_BUFFER_TOO_SMALL.  So before capturing, make one warm-up call per
+ *   shape or call elutq_reserve with the largest one; graph users who want no
+ *   library-owned memory at all use elutq_lut_gemm_ws or elutq_lut_gemm_static.
  *   Calls that share a stream are ordered; calls on different streams use
  *   different scratch buffers.
  */
 int elutq_lut_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
+
+/* Make the library-owned scratch of `stream` large enough for any call up to (M, N, K), including the
+ * staging buffers of elutq_lut_gemm_host (allocates; not during capture). */
+int elutq_reserve(int M, int N, int K, void* stream);
+
+/* Address and size of one library-owned buffer of `stream` (kind 0 = control words, 1 = X staging,
+ * 2 = Y staging, 3 = K-split partial sums); *ptr = NULL when none exists yet.  For tests and tools. */
+int elutq_scratch_address(void* stream, int kind, void** ptr, size_t* bytes);
 
 /*
  * Only the offset term of Eq. 3: Y[m,n] (+)= sum_Gi z[n,Gi] * sum_{k in Gi} X[m,k].
@@ -214,6 +244,11 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
  *   - All calls on a device share the array, which keeps the previous call's contents (nothing
  *     needs clearing: every value read was written by the same call).  Calls that overlap on the
  *     GPU, e.g. on different streams, race on it: keep them stream-ordered.
+ *   - Every M stays on the look-up kernels here (the tensor-core path needs more scratch than the array
+ *     holds), so from M = 9 on the result differs from elutq_lut_gemm's in rounding (it is the more
+ *     accurate of the two: W_hat is never rounded to fp16) and the call is slower.
+ *   - `packed` must be known to the library (packed or described in this process) before a capture
+ *     begins: an unknown address makes the call read the header with a synchronous copy.
  */
 int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
 

@@ -64,6 +64,8 @@ _SIGNATURES = {
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
+    "elutq_reserve": (c_int, [c_int, c_int, c_int, c_void_p]),
+    "elutq_scratch_address": (c_int, [c_void_p, c_int, ctypes.POINTER(c_void_p), ctypes.POINTER(c_size_t)]),
 }
 
 
@@ -253,3 +255,14 @@ def elutq_chain_status(plan, stream=None) -> int:
 
 def elutq_chain_forget(plan) -> None:
     _check(lib().elutq_chain_forget(_ptr(plan)), "elutq_chain_forget")
+
+
+def elutq_reserve(M: int, N: int, K: int, stream=None) -> None:
+    _check(lib().elutq_reserve(M, N, K, _stream(stream)), "elutq_reserve")
+
+
+def elutq_scratch_address(kind: int, stream=None):
+    """(address or None, bytes) of a library-owned scratch buffer of the stream."""
+    ptr, nb = c_void_p(0), c_size_t(0)
+    _check(lib().elutq_scratch_address(_stream(stream), kind, ctypes.byref(ptr), ctypes.byref(nb)), "elutq_scratch_address")
+    return ptr.value, nb.value

@@ -6,6 +6,7 @@
 #include <map>
 #include <mutex>
 #include <unordered_map>
+#include <vector>
 #include <utility>
 
 #include "common.cuh"
@@ -22,6 +23,9 @@ std::mutex g_mu;
 std::unordered_map<const void*, BlobMeta> g_blobs;
 
 struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
+// Buffers that a larger request has replaced.  They are kept until elutq_release_scratch: a CUDA graph captured
+// earlier holds their addresses as kernel arguments, and work enqueued earlier may still be running on them.
+std::vector<void*> g_parked;
 // keyed by (device, stream, kind): kind 0 = arrival counters (always zero between calls), 1 = X staging,
 // 2 = Y staging, 3 = K-split partial sums.  Counters live in a buffer of their own so that no other data
 // is ever written where a later call with a different shape expects zeroed counters.
@@ -54,12 +58,8 @@ int num_sms() {
     return g_num_sms[dev];
 }
 
-// Workspace layout: counters (one per row block and row-batch), rounded up to 256 bytes, then partials.
-size_t counters_bytes(int M, int N) {
-    const size_t n_rb = (size_t)(N + kTileRows - 1) / kTileRows;
-    const size_t n = n_rb * (size_t)M;   // enough for any row batching of the M rows
-    return (n * sizeof(unsigned) + 255) / 256 * 256;
-}
+// Workspace layout: a 256-byte control area (word 0 = device status), then the partial sums.
+size_t counters_bytes(int, int) { return 256; }
 size_t partials_bytes(int M, int N, int K) {
     const size_t n_rb = (size_t)(N + kTileRows - 1) / kTileRows;
     const size_t n_kc = (size_t)(K + kChunkK - 1) / kChunkK;
@@ -69,8 +69,8 @@ size_t partials_bytes(int M, int N, int K) {
     return chunks * (size_t)M * n_rb * kTileRows * sizeof(float);
 }
 
-int lookup_blob(const void* packed, int N, int K, BlobMeta* out) {
-    {
+int lookup_blob(const void* packed, int N, int K, BlobMeta* out, bool force_read = false) {
+    if (!force_read) {
         std::lock_guard<std::mutex> lk(g_mu);
         auto it = g_blobs.find(packed);
         if (it != g_blobs.end() && it->second.N == N && it->second.K == K) {
@@ -95,6 +95,8 @@ int lookup_blob(const void* packed, int N, int K, BlobMeta* out) {
 }
 
 // Library-owned scratch of at least `bytes` for (current device, stream, kind); counters zeroed on (re)allocation.
+// A buffer that has to grow is replaced, never freed (see g_parked).  Nothing is allocated while the stream is being
+// captured: the request fails with ELUTQ_ERR_BUFFER_TOO_SMALL instead (reserve before capturing).
 int get_scratch(void* stream, int kind, size_t bytes, bool zero, void** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -102,20 +104,21 @@ int get_scratch(void* stream, int kind, size_t bytes, bool zero, void** out) {
     std::lock_guard<std::mutex> lk(g_mu);
     Scratch& s = g_scratch[std::make_tuple(dev, stream, kind)];
     if (s.bytes < bytes) {
-        if (s.ptr) {
-            e = cudaFree(s.ptr);   // synchronises: no kernel can still use the old buffer
-            s.ptr = nullptr;
-            s.bytes = 0;
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing((cudaStream_t)stream, &cap);
+        if (e != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+        if (cap != cudaStreamCaptureStatusNone) return ELUTQ_ERR_BUFFER_TOO_SMALL;
         size_t want = bytes < (1u << 20) ? (1u << 20) : bytes;
-        e = cudaMalloc(&s.ptr, want);
-        if (e != cudaSuccess) { s.ptr = nullptr; return cuda_fail(e); }
-        s.bytes = want;
+        void* fresh = nullptr;
+        e = cudaMalloc(&fresh, want);
+        if (e != cudaSuccess) return cuda_fail(e);
         if (zero) {
-            e = cudaMemsetAsync(s.ptr, 0, want, (cudaStream_t)stream);
-            if (e != cudaSuccess) return cuda_fail(e);
+            e = cudaMemsetAsync(fresh, 0, want, (cudaStream_t)stream);
+            if (e != cudaSuccess) { cudaFree(fresh); return cuda_fail(e); }
         }
+        if (s.ptr) g_parked.push_back(s.ptr);
+        s.ptr = fresh;
+        s.bytes = want;
     }
     *out = s.ptr;
     return ELUTQ_OK;
@@ -171,6 +174,8 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     int st = lookup_blob(packed, N, K, &m);
     if (st != ELUTQ_OK) return st;
     if ((flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8)) && m.G != 128) return ELUTQ_ERR_UNSUPPORTED;
+    // decode-kernel variants exist for M = 1 only
+    if ((flags & (ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_CLUSTER_REDUCE)) && M > 1) return ELUTQ_ERR_UNSUPPORTED;
 
     const size_t cb = counters_bytes(M, N), pb = partials_bytes(M, N, K);
     void* counters = workspace;
@@ -204,6 +209,7 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
     else if (M >= ELUTQ_TENSOR_MIN_M && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
     else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);
+    if (ce == (int)cudaErrorNotSupported) return ELUTQ_ERR_UNSUPPORTED;
     if (ce != 0) return cuda_fail((cudaError_t)ce);
     return ELUTQ_OK;
 }
@@ -288,7 +294,7 @@ int elutq_unpack(const void* packed, int N, int K, uint8_t* planes, void* scales
 int elutq_describe(const void* packed, int N, int K, int* q, int* G) {
     if (!packed || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
     BlobMeta m;
-    int st = lookup_blob(packed, N, K, &m);
+    int st = lookup_blob(packed, N, K, &m, true);     // always the header that is there now, never a remembered one
     if (st != ELUTQ_OK) return st;
     if (q) *q = m.q;
     if (G) *G = m.G;
@@ -398,7 +404,37 @@ int elutq_release_scratch(void) {
         }
     }
     g_scratch.clear();
+    for (void* p : g_parked) {
+        cudaError_t e = cudaFree(p);
+        if (e != cudaSuccess && first == cudaSuccess) first = e;
+    }
+    g_parked.clear();
     if (first != cudaSuccess) return cuda_fail(first);
+    return ELUTQ_OK;
+}
+
+int elutq_reserve(int M, int N, int K, void* stream) {
+    if (M <= 0 || N <= 0 || K <= 0) return ELUTQ_ERR_INVALID_ARG;
+    void* p = nullptr;
+    int st = get_scratch(stream, 0, counters_bytes(M, N), true, &p);
+    if (st != ELUTQ_OK) return st;
+    const size_t pb = partials_bytes(M, N, K);
+    st = get_scratch(stream, 3, pb ? pb : 16, false, &p);
+    if (st != ELUTQ_OK) return st;
+    st = get_scratch(stream, 1, (size_t)M * K * sizeof(__half), false, &p);
+    if (st != ELUTQ_OK) return st;
+    return get_scratch(stream, 2, (size_t)M * N * sizeof(__half), false, &p);
+}
+
+int elutq_scratch_address(void* stream, int kind, void** ptr, size_t* bytes) {
+    if (!ptr || kind < 0 || kind > 3) return ELUTQ_ERR_INVALID_ARG;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::lock_guard<std::mutex> lk(g_mu);
+    auto it = g_scratch.find(std::make_tuple(dev, stream, kind));
+    *ptr = it == g_scratch.end() ? nullptr : it->second.ptr;
+    if (bytes) *bytes = it == g_scratch.end() ? 0 : it->second.bytes;
     return ELUTQ_OK;
 }
 

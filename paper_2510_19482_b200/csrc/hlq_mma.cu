@@ -154,6 +154,9 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     const bool use_planes = !(a.flags & ELUTQ_FLAG_OFFSET_ONLY);
     const bool use_offset = !(a.flags & ELUTQ_FLAG_SKIP_OFFSET);
 
+    // the blob is still the one this launch was planned for (checked before anything is allocated or read)
+    if (!blob_header_matches(a.tiles, Q, 128, a.N, a.K, a.counters)) return;
+
     // ---- set-up: tensor memory, completion barriers ---------------------------------------------
     uint32_t cta_rank = 0;                               // rank in the CTA pair (0 = leader)
     if constexpr (CG == 2) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));

@@ -308,6 +308,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemm_kernel(const GemmArgs a)
     extern __shared__ __align__(1024) uint8_t smem[];
     const float* gsum = reinterpret_cast<const float*>(smem + C::TABLE_BYTES);
 
+    if (!blob_header_matches(a.tiles, Q, G, a.N, a.K, a.counters)) return;   // before any tile is read
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
     const int bid = blockIdx.x;

@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
     extern __shared__ __align__(1024) uint8_t smem[];
     const float* gsum = reinterpret_cast<const float*>(smem + kTableBytes);
 
+    if (!blob_header_matches(a.tiles, Q, G, a.N, a.K, a.counters)) return;   // before any tile is read
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int h = lane >> 4, l = lane & 15;
     const int bid = blockIdx.x;
@@ -161,6 +162,7 @@ __global__ void __launch_bounds__(kThreads, 1) lut_gemv_kernel(const GemmArgs a)
 __global__ void __launch_bounds__(256) lut_finalize_kernel(const GemmArgs a, const int n_chunks, const int col0, const int cols) {
     grid_launch_dependents();
     grid_dependency_wait();
+    if (a.counters != nullptr && __ldcg(a.counters) != 0u) return;   // the main kernel refused the blob: no partial sums, no Y
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)a.M * cols) return;
     const int m = (int)(idx / cols), row = col0 + (int)(idx % cols);
@@ -178,6 +180,7 @@ __global__ void __launch_bounds__(256) lut_finalize_parts_kernel(const GemmArgs 
     __shared__ float sub[8][32];
     grid_launch_dependents();
     grid_dependency_wait();
+    if (a.counters != nullptr && __ldcg(a.counters) != 0u) return;   // the main kernel refused the blob: no partial sums, no Y
     const int lane = threadIdx.x & 31, part = threadIdx.x >> 5, parts = blockDim.x >> 5;
     const long long idx = (long long)blockIdx.x * 32 + lane;
     const bool live = idx < (long long)a.M * cols;

@@ -93,6 +93,7 @@ __global__ void pack_params_kernel(const uint16_t* __restrict__ scales, const ui
 
 // One thread per (plane j, row n, byte-column cg): expands a packed byte to 8 uint8 {0,1}.
 __global__ void unpack_planes_kernel(const uint8_t* __restrict__ tiles, uint8_t* __restrict__ planes, Geo g) {
+    if (!blob_header_matches(tiles, g.q, g.G, g.N, g.K, nullptr)) return;   // before any tile is read
     const int cols = g.K / 8;
     const long long total = (long long)g.q * g.N * cols;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -120,6 +121,7 @@ __global__ void unpack_planes_kernel(const uint8_t* __restrict__ tiles, uint8_t*
 // One thread per (row n, group gi, component): copies one fp16 parameter back.
 __global__ void unpack_params_kernel(const uint8_t* __restrict__ tiles, uint16_t* __restrict__ scales,
                                      uint16_t* __restrict__ offsets, Geo g) {
+    if (!blob_header_matches(tiles, g.q, g.G, g.N, g.K, nullptr)) return;   // before any tile is read
     const int Gn = g.K / g.G;
     const long long total = (long long)g.N * Gn * (g.q + 1);
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;

@@ -74,3 +74,33 @@ def test_pointer_validation_happens_before_any_launch():
     assert L.elutq_forget(None) == -1
     assert elutq.elutq_launch_count() == before
     assert elutq.elutq_status_string(-4) == "buffer too small"
+
+
+def test_chain_argument_validation_happens_on_the_host():
+    L = elutq.lib()
+    out = ctypes.c_size_t(0)
+    before = elutq.elutq_launch_count()
+    good = (elutq.GemvCall * 2)(elutq.GemvCall(16, 16, 16, 64, 1024, 0), elutq.GemvCall(32, 32, 32, 4096, 4096, 0x4))
+    assert L.elutq_chain_plan_bytes(good, 2, ctypes.byref(out)) == 0
+    # control block + counters + descriptors + CTA shares + three scratch regions of 8 chunks x 4096 rows x 8 bytes
+    assert out.value > 3 * 8 * 4096 * 8
+    assert L.elutq_chain_plan_bytes(None, 2, ctypes.byref(out)) == -1
+    assert L.elutq_chain_plan_bytes(good, 0, ctypes.byref(out)) == -1
+    assert L.elutq_chain_plan_bytes(good, 5000, ctypes.byref(out)) == -1
+    bad = (elutq.GemvCall * 1)(elutq.GemvCall(16, 16, 0, 64, 1024, 0))
+    assert L.elutq_chain_plan_bytes(bad, 1, ctypes.byref(out)) == -1          # null Y
+    bad = (elutq.GemvCall * 1)(elutq.GemvCall(8, 16, 16, 64, 1024, 0))
+    assert L.elutq_chain_plan_bytes(bad, 1, ctypes.byref(out)) == -3          # X not 16-byte aligned
+    bad = (elutq.GemvCall * 1)(elutq.GemvCall(16, 16, 16, 64, 1024, 0x1))
+    assert L.elutq_chain_plan_bytes(bad, 1, ctypes.byref(out)) == -5          # term flags are not offered by the chain
+    bad = (elutq.GemvCall * 1)(elutq.GemvCall(16, 16, 16, 64, 1024, 0x800))
+    assert L.elutq_chain_plan_bytes(bad, 1, ctypes.byref(out)) == -1          # unknown flag
+    assert L.elutq_chain_plan(good, 2, None, 0, None) == -1
+    assert L.elutq_chain_plan(good, 2, 128, 1 << 30, None) == -3              # plan buffer not 256-byte aligned
+    assert L.elutq_chain_plan(good, 2, 256, 16, None) == -4                   # plan buffer too small
+    assert L.elutq_chain_run(None, 2, None) == -1
+    assert L.elutq_chain_run(256, 2, None) == -2                              # a buffer that was never planned
+    assert L.elutq_chain_status(None, None, None) == -1
+    assert L.elutq_reserve(0, 16, 512, None) == -1
+    assert L.elutq_scratch_address(None, 9, None, None) == -1
+    assert elutq.elutq_launch_count() == before
