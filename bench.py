@@ -7,12 +7,18 @@ twelve M = 1 decode linears of the LLaMA-3.1-8B shapes at q in {2,3,4}, G = 128.
 printed by rank 0:
 
   value       achieved GB/s = algorithmic bytes of the step (bit-planes + fp16 scales + fp16 offsets +
-              X + Y, summed over the calls) / device time, inputs resident in HBM, the step replayed
-              from a CUDA graph of C-ABI calls; the working set of a step exceeds the L2 capacity
+              X + Y, summed over the calls) / device time, inputs resident in HBM.  M = 1 workloads run
+              the step through the chained decode entry (elutq_chain_run: the list of calls in one
+              persistent launch per bit-width); the same step as separate elutq_lut_gemm calls replayed
+              from a CUDA graph is timed beside it (`secondary`).  The working set of a step exceeds
+              the L2 capacity
   e2e         the same metric through elutq_lut_gemm_host: X copied from pinned host memory and Y copied
               back inside the timed region, every call
   roofline    achieved / measured HBM copy bandwidth for the decode kernel
   cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample of the same workload
+  secondary   short same-run measurements of the other configurations (70B decode, one 2-bit GEMV
+              isolated / L2-hot, small-batch sweep, prefill, 32-layer stack), each with its own roofline
+              fraction; their inputs are drawn on the device (same shapes and distributions)
 
 `--impl reference` times the oracle alone (the only reference there is: the paper ships no code).
 """
@@ -243,6 +249,218 @@ def aggregate_value(step_bytes: int, world: int, ms_per_step: float) -> float:
     return world * step_bytes / (ms_per_step * 1e-3) / 1e9
 
 
+MIN_TIMED_SECONDS = 0.2      # the timed region replays the step until it lasts at least this long
+
+
+def _device_layer(torch, elutq, c, gen):
+    """Packed layer with inputs drawn on the device (timing-only: same shapes and distributions as the recipe)."""
+    Gn = c.K // c.G
+    planes = torch.randint(0, 2, (c.q, c.N, c.K), dtype=torch.uint8, device="cuda", generator=gen)
+    scales = (torch.randn((c.N, Gn, c.q), device="cuda", generator=gen) * 0.02).abs().to(torch.float16)
+    offsets = (torch.randn((c.N, Gn), device="cuda", generator=gen) * 0.01).to(torch.float16)
+    packed = elutq.elutq_pack(planes, scales, offsets, c.q, c.G, c.N, c.K)
+    torch.cuda.synchronize()
+    return packed
+
+
+class _Runner:
+    """One step of a call list, replayed over rotating copies of its buffers: as one chain (M = 1 lists) or as a
+    CUDA graph of separate C-ABI calls."""
+
+    def __init__(self, torch, elutq, sets, mode, stream, flags=0):
+        self.torch, self.elutq, self.sets, self.mode, self.stream = torch, elutq, sets, mode, stream
+        self.copies = len(sets)
+        self.n = len(sets[0])
+        self.plans, self.graphs = [], []
+        with torch.cuda.stream(stream):
+            if mode == "chain":
+                for st in sets:
+                    self.plans.append(elutq.elutq_chain_plan(
+                        [(l["X"], l["packed"], l["Y"], l["call"].N, l["call"].K) for l in st], stream=stream))
+                self.one(0)
+                stream.synchronize()
+                c0 = elutq.elutq_launch_count()
+                self.one(0)
+                self.launches_per_step = int(elutq.elutq_launch_count() - c0)
+            else:
+                self._eager(0, flags)          # allocates the library's scratch before capture
+                stream.synchronize()
+                c0 = elutq.elutq_launch_count()
+                self._eager(0, flags)
+                self.launches_per_step = int(elutq.elutq_launch_count() - c0)
+                stream.synchronize()
+                for r in range(self.copies):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        self._eager(r, flags)
+                    self.graphs.append(g)
+            stream.synchronize()
+
+    def _eager(self, r, flags):
+        for l in self.sets[r]:
+            c = l["call"]
+            if flags:
+                self.elutq.elutq_lut_gemm_ws(l["X"], l["packed"], l["Y"], c.M, c.N, c.K, flags, l["ws"], stream=self.stream)
+            else:
+                self.elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K, stream=self.stream)
+
+    def one(self, i):
+        r = i % self.copies
+        if self.mode == "chain":
+            self.elutq.elutq_chain_run(self.plans[r], self.n, stream=self.stream)
+        else:
+            self.graphs[r].replay()
+
+    def timed(self, steps, warmup, barrier=None):
+        """Device time (ms) of exactly steps * reps steps; reps makes the region last MIN_TIMED_SECONDS."""
+        torch = self.torch
+        with torch.cuda.stream(self.stream):
+            for i in range(warmup):
+                self.one(i)
+            self.stream.synchronize()
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            probe = max(3, min(steps, 20))
+            p0.record(self.stream)
+            for i in range(probe):
+                self.one(i)
+            p1.record(self.stream)
+            self.stream.synchronize()
+            per = max(p0.elapsed_time(p1) / probe, 1e-4)
+            reps = max(1, int(-(-MIN_TIMED_SECONDS * 1e3 // (per * steps))))
+            if barrier:
+                barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.time()
+            e0.record(self.stream)
+            for i in range(steps * reps):
+                self.one(i)
+            e1.record(self.stream)
+            if barrier:
+                barrier()
+            self.stream.synchronize()
+            t1 = time.time()
+            return e0.elapsed_time(e1), reps, t0, t1
+
+    def status(self):
+        if self.mode == "chain":
+            return max(self.elutq.elutq_chain_status(p, stream=self.stream) for p in self.plans)
+        return self.elutq.elutq_device_status(self.stream)
+
+    def close(self):
+        for p in self.plans:
+            self.elutq.elutq_chain_forget(p)
+        self.plans, self.graphs = [], []
+
+
+def _make_sets(torch, elutq, layers, l2_bytes, flags=0, max_copies=8):
+    """Rotating copies of the packed layers (and X / Y) so that >= 3x L2 is touched between two uses of a copy."""
+    working_set = sum(l["packed"].numel() for l in layers)
+    copies = max(1, min(max_copies, -(-3 * l2_bytes // max(working_set, 1))))
+    if copies * working_set > (24 << 30):
+        copies = 1
+    sets = [layers]
+    for _ in range(1, copies):
+        dup = []
+        for l in layers:
+            c = l["call"]
+            d = dict(l)
+            d["packed"] = l["packed"].clone()
+            elutq.elutq_describe(d["packed"], c.N, c.K)
+            d["X"] = l["X"].clone()
+            d["Y"] = torch.empty_like(l["Y"])
+            if flags:
+                d["ws"] = torch.empty_like(l["ws"])
+                elutq.elutq_workspace_init(d["ws"])
+            dup.append(d)
+        sets.append(dup)
+    torch.cuda.synchronize()
+    return sets, copies, working_set
+
+
+def _secondary(torch, elutq, name, stream, l2_bytes, hbm_peak, tensor_peak, device_index):
+    """Short same-run measurement of another configuration; inputs drawn on the device."""
+    calls = _calls(name)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234)
+    cache = {}
+    layers = []
+    for c in calls:
+        key = (c.q, c.G, c.N, c.K) if name != "cfg4_stack" else (c.name,)
+        if key not in cache:
+            cache[key] = _device_layer(torch, elutq, c, gen)
+        X = torch.randn((c.M, c.K), device="cuda", generator=gen).to(torch.float16)
+        layers.append(dict(call=c, packed=cache[key], X=X, Y=torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")))
+    step_bytes = _bytes_of(calls)
+    all_m1 = all(c.M == 1 for c in calls)
+    tensor = all(c.M >= 9 and c.G == 128 for c in calls)
+    # distinct blobs are shared between the calls of a step here, so rotate whole copies only while they are small
+    distinct = sum(t.numel() for t in cache.values())
+    out = {"workload": WORKLOAD_NAMES[name], "calls_per_step": len(calls), "algorithmic_bytes_per_step": step_bytes,
+           "data": "synthetic, drawn on the device (timing only)"}
+    results = {}
+    for mode in (("chain", "graph") if all_m1 else ("graph",)):
+        sets = [layers]
+        copies = 1
+        if distinct < 3 * l2_bytes:
+            copies = max(1, min(8, -(-3 * l2_bytes // max(distinct, 1))))
+            sets = [layers]
+            for _ in range(1, copies):
+                dup_cache = {k: v.clone() for k, v in cache.items()}
+                dup = []
+                for l in layers:
+                    c = l["call"]
+                    key = (c.q, c.G, c.N, c.K) if name != "cfg4_stack" else (c.name,)
+                    elutq.elutq_describe(dup_cache[key], c.N, c.K)
+                    dup.append(dict(call=c, packed=dup_cache[key], X=l["X"].clone(), Y=torch.empty_like(l["Y"])))
+                sets.append(dup)
+        runner = _Runner(torch, elutq, sets, mode, stream)
+        sampler = ClockSampler(device_index)
+        ms, reps, t0, t1 = runner.timed(10, 5)
+        clocks = sampler.stop(t0, t1)
+        ms_step = ms / (10 * reps)
+        r = {"ms_per_step": ms_step, "us_per_call_mean": ms_step * 1e3 / len(calls), "launches_per_step": runner.launches_per_step,
+             "device_status": runner.status(), "clocks": clocks,
+             "l2": f"{copies} rotating copies of the distinct layers ({copies * distinct / l2_bytes:.1f}x L2)"}
+        if tensor:
+            tf = sum(2.0 * c.M * c.N * c.K for c in calls) / (ms_step * 1e-3) / 1e12
+            r.update({"bound": "tensor", "achieved": tf, "unit": "TFLOP/s", "peak": tensor_peak, "frac": tf / tensor_peak})
+        else:
+            gbs = step_bytes / (ms_step * 1e-3) / 1e9
+            r.update({"bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": hbm_peak, "frac": gbs / hbm_peak})
+        results["chain (elutq_chain_run)" if mode == "chain" else "separate calls (CUDA graph)"] = r
+        runner.close()
+        del runner, sets
+    out["runs"] = results
+    if name == "cfg0":
+        # one 2-bit GEMV, isolated (one launch between two synchronisations) and L2-hot (the same blob again and again):
+        # labelled figures, not HBM-roofline figures
+        l = layers[0]
+        c = l["call"]
+        with torch.cuda.stream(stream):
+            ts = []
+            for _ in range(60):
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                stream.synchronize()
+                a0.record(stream)
+                elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K, stream=stream)
+                a1.record(stream)
+                stream.synchronize()
+                ts.append(a0.elapsed_time(a1) * 1e3)
+            ts = sorted(ts[10:])
+            hot = _Runner(torch, elutq, [layers], "graph", stream)
+            ms, reps, _, _ = hot.timed(50, 10)
+            out["isolated_call_us_median"] = ts[len(ts) // 2]
+            out["l2_hot_us_per_call"] = ms * 1e3 / (50 * reps)
+            out["isolated_note"] = "one elutq_lut_gemm between two stream synchronisations (launch latency included); " \
+                                   "L2-hot: the same 5 MB blob replayed back to back from a graph; neither is an HBM figure"
+            hot.close()
+    for t in cache.values():
+        elutq.elutq_forget(t)
+    del layers, cache
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args) -> None:
     import torch
     import torch.distributed as dist
@@ -277,7 +495,6 @@ def run_cuda(args) -> None:
         layers.append(dict(call=c, packed=packed, X=Xh.cuda(), Y=torch.empty((c.M, c.N), dtype=torch.float16, device="cuda"),
                            Xh=Xh, Yh=Yh))
     step_bytes = _bytes_of(calls)
-    working_set = sum(l["packed"].numel() for l in layers)
 
     if args.flags:
         # variant runs go through the caller-workspace entry point, one workspace per call
@@ -290,112 +507,82 @@ def run_cuda(args) -> None:
     # HBM-cold protocol: consecutive steps rotate over distinct copies of the packed layers (and of X / Y) so
     # that the bytes touched between two uses of the same copy are at least 3x the L2 capacity
     l2_bytes = int(getattr(torch.cuda.get_device_properties(local_rank), "L2_cache_size", 126 << 20))
-    copies = max(1, min(8, -(-3 * l2_bytes // max(working_set, 1))))
-    if copies * working_set > (16 << 30):
-        copies = 1
-    if os.environ.get("ELUTQ_BENCH_COPIES"):          # experiments: e.g. 1 keeps a small working set L2-resident
-        copies = max(1, int(os.environ["ELUTQ_BENCH_COPIES"]))
-    layer_sets = [layers]
-    for _ in range(1, copies):
-        dup = []
-        for l in layers:
-            c = l["call"]
-            d = dict(l)
-            d["packed"] = l["packed"].clone()
-            elutq.elutq_describe(d["packed"], c.N, c.K)
-            d["X"] = l["X"].clone()
-            d["Y"] = torch.empty_like(l["Y"])
-            if args.flags:
-                d["ws"] = torch.empty_like(l["ws"])
-                elutq.elutq_workspace_init(d["ws"])
-            dup.append(d)
-        layer_sets.append(dup)
-    torch.cuda.synchronize()
-
-    def step(r=0):
-        for l in layer_sets[r]:
-            c = l["call"]
-            if args.flags:
-                elutq.elutq_lut_gemm_ws(l["X"], l["packed"], l["Y"], c.M, c.N, c.K, args.flags, l["ws"])
-            else:
-                elutq.elutq_lut_gemm(l["X"], l["packed"], l["Y"], c.M, c.N, c.K)
-
-    def step_host():
-        for l in layers:
-            c = l["call"]
-            elutq.elutq_lut_gemm_host(l["Xh"], l["packed"], l["Yh"], c.M, c.N, c.K)
+    layer_sets, copies, working_set = _make_sets(torch, elutq, layers, l2_bytes, args.flags)
 
     stream = torch.cuda.Stream()
+    use_chain = all(c.M == 1 for c in calls) and not args.flags and not args.no_chain and not args.no_graph
+    peak, peak_src = _peaks()
+    tpeak, tsrc = _tensor_peak()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if args.no_graph:
+        # plain stream of C-ABI calls (no graph, no chain): a debugging mode
+        class _Eager(_Runner):
+            def __init__(self):
+                self.torch, self.elutq, self.sets, self.mode, self.stream = torch, elutq, layer_sets, "eager", stream
+                self.copies, self.n, self.plans, self.graphs = copies, len(layers), [], []
+                with torch.cuda.stream(stream):
+                    c0 = elutq.elutq_launch_count()
+                    self._eager(0, args.flags)
+                    stream.synchronize()
+                    self.launches_per_step = int(elutq.elutq_launch_count() - c0)
+
+            def one(self, i):
+                self._eager(i % self.copies, args.flags)
+        main = _Eager()
+    else:
+        main = _Runner(torch, elutq, layer_sets, "chain" if use_chain else "graph", stream, args.flags)
+
+    # ---- device-resident timing -------------------------------------------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms, reps, t_wall0, t_wall1 = main.timed(args.steps, args.warmup, barrier)
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    launches = main.launches_per_step * args.steps * reps
+    main_status = main.status()
+
+    # ---- spread of single steps (separate pass; the headline above is the timed region) --------------
     with torch.cuda.stream(stream):
-        step()              # allocates the library's scratch before capture
-        step_host()
-        stream.synchronize()
-        graph = None
-        graphs = []
-        if not args.no_graph:
-            for r in range(copies):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    step(r)
-                graphs.append(g)
-            graph = graphs[0]
-
-        def run(n):
-            for i in range(n):
-                if graph is not None:
-                    graphs[i % copies].replay()
-                else:
-                    step(i % copies)
-
-        def barrier():
-            torch.cuda.synchronize()
-            if world > 1:
-                dist.barrier()
-            torch.cuda.synchronize()
-
-        # ---- device-resident timing -------------------------------------------------------------
-        sampler = ClockSampler(local_rank) if rank == 0 else None
-        run(args.warmup)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        launches_before = elutq.elutq_launch_count()
-        t_wall0 = time.time()
-        e0.record()
-        run(args.steps)
-        e1.record()
-        barrier()
-        t_wall1 = time.time()
-        ms = e0.elapsed_time(e1)
-        clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-        if graph is not None:
-            # a graph replay launches what one eager step launches: count the library's kernel launches of one step
-            c0 = elutq.elutq_launch_count()
-            step(0)
-            stream.synchronize()
-            launches = int(elutq.elutq_launch_count() - c0) * args.steps
-        else:
-            launches = int(elutq.elutq_launch_count() - launches_before)
-
-        # ---- spread of single steps (separate pass; the headline above is the K-step region) --------------
         spread_n = max(3, min(args.steps, 200))
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(spread_n + 1)]
-        evs[0].record()
+        evs[0].record(stream)
         for i in range(spread_n):
-            if graph is not None:
-                graphs[i % copies].replay()
-            else:
-                step(i % copies)
-            evs[i + 1].record()
-        torch.cuda.synchronize()
+            main.one(i)
+            evs[i + 1].record(stream)
+        stream.synchronize()
         singles = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(spread_n))
         ms_median, ms_min = singles[len(singles) // 2], singles[0]
 
-        # ---- end to end through the host entry point ---------------------------------------------
-        # (the same launch mode as above: a CUDA graph of the public host-buffer calls, whose copy nodes read the
-        #  pinned inputs and write the pinned outputs on every replay)
-        e2e_steps = max(1, min(args.steps, 200))
+    # ---- the same step as separate calls (when the headline is the chain) ------------------------------
+    separate = None
+    graph_runner = main if (not use_chain and not args.no_graph) else None
+    if use_chain:
+        graph_runner = _Runner(torch, elutq, layer_sets, "graph", stream)
+        sms, sreps, _, _ = graph_runner.timed(min(args.steps, 200), min(args.warmup, 20))
+        sms_step = sms / (min(args.steps, 200) * sreps)
+        sg = step_bytes / (sms_step * 1e-3) / 1e9
+        separate = {"ms_per_step": sms_step, "us_per_call_mean": sms_step * 1e3 / len(calls), "achieved": sg, "unit": "GB/s",
+                    "frac": sg / peak, "launches_per_step": graph_runner.launches_per_step,
+                    "launch": "the same step as separate elutq_lut_gemm calls, CUDA graph, programmatic dependent launch"}
+
+    # ---- end to end through the host entry point ---------------------------------------------
+    # (a CUDA graph of the public host-buffer calls, whose copy nodes read the pinned inputs and write the pinned
+    #  outputs on every replay)
+    def step_host():
+        for l in layers:
+            c = l["call"]
+            elutq.elutq_lut_gemm_host(l["Xh"], l["packed"], l["Yh"], c.M, c.N, c.K, stream=stream)
+
+    e2e_steps = max(1, min(args.steps, 200))
+    with torch.cuda.stream(stream):
+        step_host()
+        stream.synchronize()
         host_graph = None
-        if graph is not None:
+        if not args.no_graph:
             host_graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(host_graph, stream=stream):
                 step_host()
@@ -410,10 +597,10 @@ def run_cuda(args) -> None:
             run_host()
         barrier()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        h0.record()
+        h0.record(stream)
         for _ in range(e2e_steps):
             run_host()
-        h1.record()
+        h1.record(stream)
         barrier()
         ms_host = h0.elapsed_time(h1)
 
@@ -421,19 +608,20 @@ def run_cuda(args) -> None:
         # (the extra call reads its own copy of the packed layer, so it is HBM-cold like the others and
         #  does not warm the L2 for the step's own call)
         per_call = []
-        if rank == 0 and not args.no_per_call and graph is not None:
-            reps = max(20, min(args.steps, 300))
+        if rank == 0 and not args.no_per_call and graph_runner is not None:
+            reps_pc = max(20, min(args.steps, 300))
+            graph = graph_runner.graphs[0]
 
             def time_graph(g):
                 for _ in range(3):
                     g.replay()
                 a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a0.record()
-                for _ in range(reps):
+                a0.record(stream)
+                for _ in range(reps_pc):
                     g.replay()
-                a1.record()
-                torch.cuda.synchronize()
-                return a0.elapsed_time(a1) * 1e3 / reps
+                a1.record(stream)
+                stream.synchronize()
+                return a0.elapsed_time(a1) * 1e3 / reps_pc
 
             seen = {}
             for l in layers:
@@ -447,17 +635,36 @@ def run_cuda(args) -> None:
                 Y2 = torch.empty_like(l["Y"])
                 g2 = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g2, stream=stream):
-                    elutq.elutq_lut_gemm(l["X"], clone, Y2, c.M, c.N, c.K)
-                    step()
+                    elutq.elutq_lut_gemm(l["X"], clone, Y2, c.M, c.N, c.K, stream=stream)
+                    graph_runner._eager(0, 0)
                 t_base = time_graph(graph)
                 us = max(time_graph(g2) - t_base, 0.0)
                 b = workloads.algorithmic_bytes(c.M, c.N, c.K, c.q, c.G)
                 per_call.append({"name": key[0], "q": c.q, "M": c.M, "N": c.N, "K": c.K, "us": round(us, 3),
                                  "GBps": round(b / max(us, 1e-3) / 1e3, 1),
-                                 "frac_of_hbm_peak": round(b / max(us, 1e-3) / 1e3 / _peaks()[0], 3),
-                                 "tflop_eq": round(2.0 * c.M * c.N * c.K / max(us, 1e-3) / 1e6, 3)})
+                                 "frac_of_hbm_peak": round(b / max(us, 1e-3) / 1e3 / peak, 3),
+                                 "tflop_eq": round(2.0 * c.M * c.N * c.K / max(us, 1e-3) / 1e6, 3),
+                                 "how": "marginal time of one extra separate call inside the graph-replayed step"})
                 elutq.elutq_forget(clone)
                 del g2, clone, Y2
+
+    # ---- the other configurations, measured briefly in the same run -----------------------------------
+    secondary = []
+    if rank == 0 and args.workload == "cfg1" and not args.no_secondary and not args.flags:
+        main.close()
+        if graph_runner is not None and graph_runner is not main:
+            graph_runner.close()
+        del main, graph_runner, layer_sets, host_graph
+        for l in layers:
+            elutq.elutq_forget(l["packed"])
+        layers_meta = [l["call"] for l in layers]
+        del layers
+        torch.cuda.empty_cache()
+        for name in ("cfg3", "cfg0", "cfg2", "cfg4_prefill", "cfg4_stack"):
+            try:
+                secondary.append(_secondary(torch, elutq, name, stream, l2_bytes, peak, tpeak, local_rank))
+            except Exception as ex:      # a failed side measurement must not lose the headline
+                secondary.append({"workload": WORKLOAD_NAMES[name], "error": repr(ex)})
 
     # ---- reduce over ranks ---------------------------------------------------------------------
     ms, ms_host = max_over_ranks([ms, ms_host])
@@ -466,10 +673,9 @@ def run_cuda(args) -> None:
             dist.destroy_process_group()
         return
 
-    ms_per_step = ms / args.steps
+    ms_per_step = ms / (args.steps * reps)
     value = aggregate_value(step_bytes, world, ms_per_step)
     e2e_value = aggregate_value(step_bytes, world, ms_host / e2e_steps)
-    peak, peak_src = _peaks()
     per_gpu = step_bytes / (ms_per_step * 1e-3) / 1e9
     traffic = _traffic_note() if args.workload == "cfg1" and not args.flags else None
     roofline = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s", "frac": per_gpu / peak,
@@ -480,7 +686,6 @@ def run_cuda(args) -> None:
     if tensor_path:
         # every call of the step is a dense contraction on the tensor cores: report FLOP/s against the measured
         # GEMM peak (the sustained figure, since the kernels are timed inside a long step)
-        tpeak, tsrc = _tensor_peak()
         tf = sum(2.0 * c.M * c.N * c.K for c in calls) / (ms_per_step * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak,
                     "peak_source": tsrc, "traffic": None,
@@ -489,16 +694,15 @@ def run_cuda(args) -> None:
     # ---- CPU baseline: the oracle on a bounded sample of the same workload -------------------------
     cpu = None
     if not args.no_cpu_baseline:
-        # a short probe sizes the sample for about 15 s of CPU work (bounded below and above)
-        probe_rows = 256
-        _, probe_dt = _time_oracle(_oracle_sample(calls, probe_rows, seed=0), 1, 0)
-        rows = int(max(256, min(4096, probe_rows * 15.0 / max(probe_dt, 1e-3))))   # generation time bounds it too
-        sample = _oracle_sample(calls, rows, seed=0)
-        gbs, dt = _time_oracle(sample, 1, 0)
-        cpu = {"value": gbs, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
-               "sample": f"first {rows} output rows (or all, where a layer has fewer) of each of the {len(calls)} layers, "
-                         f"one pass ({dt:.1f} s)"}
+        cpu = _cpu_baseline(calls)
 
+    if use_chain:
+        launch_desc = ("chained decode entry: elutq_chain_run, one persistent launch per run of equal bit-width "
+                       f"({main_launches_per_step(launches, args.steps * reps)} per step), calls ordered as if run one after another")
+    elif args.no_graph:
+        launch_desc = "stream of C-ABI calls"
+    else:
+        launch_desc = "CUDA graph of C-ABI calls, programmatic dependent launch"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -506,25 +710,64 @@ def run_cuda(args) -> None:
         "config": {"workload": WORKLOAD_NAMES[args.workload], "calls_per_step": len(calls),
                    "us_per_call_mean": ms_per_step * 1e3 / len(calls),
                    "algorithmic_bytes_per_step": step_bytes, "packed_working_set_bytes": working_set,
+                   "timed_region": f"{args.steps} steps x {reps} replays = {args.steps * reps} steps in {ms:.1f} ms",
                    "ms_per_step_median": ms_median, "ms_per_step_min": ms_min,
                    "l2": (f"no flush: consecutive steps rotate over {copies} distinct copies of the packed layers, "
                           f"{copies * working_set / l2_bytes:.1f}x the {l2_bytes >> 20} MiB L2 between two uses of a copy")
                          if copies * working_set >= 3 * l2_bytes
                          else "working set below 3x L2 (partly L2-hot number, not an HBM figure)",
-                   "launch": "CUDA graph of C-ABI calls, programmatic dependent launch" if graph is not None else "stream of C-ABI calls",
+                   "launch": launch_desc, "device_status": main_status,
                    "parallelism": "replicas only (independent batch per rank, no collective)"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(2 * c.M * c.K for c in calls),
-                "d2h_bytes_per_step": sum(2 * c.M * c.N for c in calls)},
+                "d2h_bytes_per_step": sum(2 * c.M * c.N for c in calls),
+                "how": "elutq_lut_gemm_host per call (pinned host X in, Y out), CUDA graph"},
         "gpu_launches": launches,
         "clocks": clocks,
         "cpu_baseline": cpu,
+        "separate_calls": separate,
         "per_call": per_call,
+        "secondary": secondary,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def main_launches_per_step(launches: int, steps: int) -> int:
+    return launches // max(steps, 1)
+
+
+def _cpu_baseline(calls):
+    """The oracle as it stands on a bounded sample: all cores, one thread, and one M = 32 call."""
+    # a short probe sizes the sample for about 12 s of CPU work (bounded below and above)
+    probe_rows = 256
+    _, probe_dt = _time_oracle(_oracle_sample(calls, probe_rows, seed=0), 1, 0)
+    rows = int(max(256, min(12288, probe_rows * 12.0 / max(probe_dt, 1e-3))))   # generation time bounds it too
+    sample = _oracle_sample(calls, rows, seed=0)
+    gbs, dt = _time_oracle(sample, 1, 0)
+    cpu = {"value": gbs, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+           "sample": f"first {rows} output rows (or all, where a layer has fewer) of each of the {len(calls)} layers, "
+                     f"one pass ({dt:.1f} s)"}
+    try:
+        from threadpoolctl import threadpool_limits
+        small = _oracle_sample(calls, max(64, rows // 8), seed=0)
+        with threadpool_limits(limits=1):
+            g1, d1 = _time_oracle(small, 1, 0)
+        cpu["single_thread"] = {"value": g1, "unit": UNIT, "cores": 1,
+                                "sample": f"first {max(64, rows // 8)} output rows of each layer, one pass ({d1:.1f} s)"}
+    except Exception as ex:
+        cpu["single_thread"] = {"error": repr(ex)}
+    try:
+        c = workloads.shapes.Call("o", 32, 4096, 4096, 2)
+        m32 = _oracle_sample([c], 2048, seed=0)
+        g32, d32 = _time_oracle(m32, 1, 0)
+        cpu["m32"] = {"value": g32, "unit": UNIT, "cores": _oracle_threads(), "tflop_eq": 2.0 * 32 * 2048 * 4096 / d32 / 1e12,
+                      "sample": f"M = 32, first 2048 rows of the 4096 x 4096 2-bit layer, one pass ({d32:.1f} s)"}
+    except Exception as ex:
+        cpu["m32"] = {"error": repr(ex)}
+    return cpu
 
 
 def run_fit(args) -> None:
@@ -589,6 +832,10 @@ def main() -> None:
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-call", action="store_true")
+    ap.add_argument("--no-chain", action="store_true", help="time M = 1 steps as separate calls only")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the short measurements of the other configurations")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="the timed region replays the K steps until it lasts this long (0: exactly K steps; profiler captures)")
     args = ap.parse_args()
     if args.workload.startswith("fit:"):
         args.steps = args.steps or 5
@@ -605,6 +852,7 @@ def main() -> None:
         args.warmup = 200 if args.impl == "cuda" else 3
     if args.warmup < 3:
         args.warmup = 3
+    globals()["MIN_TIMED_SECONDS"] = max(0.0, args.min_seconds)
     if args.impl == "reference":
         run_reference(args)
     else:
