@@ -101,6 +101,24 @@ def scale_term(X, planes, scales, G, row_block: int = 1024) -> np.ndarray:
     return matmul(X, planes, scales, zero, G, row_block)
 
 
+def magnitude_bound(X: np.ndarray, scales: np.ndarray, offsets: np.ndarray, G: int) -> np.ndarray:
+    """A[m,n] = sum_Gi a[n,Gi] * sum_{k in Gi} |X[m,k]|  with  a = |z + (1/2) sum_j s_j| + (1/2) sum_j |s_j|.
+
+    In the +-1 form of Appendix D every weight of a group is  z^ + sum_j (+-) s_j / 2  with z^ = z + (1/2) sum_j s_j,
+    so a[n,Gi] bounds the magnitude of every weight of the group AND of every intermediate sum met when the terms
+    are added one by one, whatever the bit-planes are: A >= |X| |W_hat|^T element-wise.  The parity tests use A as
+    the scale of element-wise error bounds (each rounding of a path costs at most its unit roundoff times A).
+    Independent of the planes, cost O(M N K / G).  Returns fp64 [M,N].
+    """
+    X64 = np.abs(np.asarray(X, dtype=np.float64))
+    M, K = X64.shape
+    s = np.asarray(scales, dtype=np.float64)
+    z = np.asarray(offsets, dtype=np.float64)
+    a = np.abs(z + 0.5 * s.sum(axis=2)) + 0.5 * np.abs(s).sum(axis=2)      # [N, K/G]
+    S = X64.reshape(M, K // G, G).sum(axis=2)                              # [M, K/G]
+    return S @ a.T
+
+
 def to_fp16(Y: np.ndarray) -> np.ndarray:
     """Round an fp64 result once to fp16 (round-to-nearest-even), as the library's output does."""
     return np.asarray(Y, dtype=np.float64).astype(np.float16)

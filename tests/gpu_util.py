@@ -40,3 +40,25 @@ def gemm_f16(X: np.ndarray, packed, N: int, K: int) -> np.ndarray:
     elutq.elutq_lut_gemm(x_dev(X), packed, Y, M, N, K)
     torch.cuda.synchronize()
     return Y.cpu().numpy()
+
+
+def assert_elementwise(y, ref, A, q: int, K: int, tensor_path: bool, out_f16: bool, where="") -> None:
+    """Element-wise bound over ALL outputs (a norm can hide one wrong element in a large result).
+
+    A = oracle.hlq.magnitude_bound(X, scales, offsets, G) bounds |X| |W_hat|^T and every intermediate of the +-1
+    form.  Roundings of the paths, each at most its unit roundoff times A (worst case, all errors aligned):
+      look-up kernels   fp32 table entries and fp32 accumulation over K terms      K * 2^-24 * A
+      tensor-core path  W_hat rebuilt in fp16: z^ rounded once, one rounding per plane add   (q + 1) * 2^-11 * A
+                        then fp32 accumulation in tensor memory                    K * 2^-23 * A
+      fp16 output       one more rounding of the result                            2^-11 * |y|
+    """
+    import numpy as np
+    y64 = np.asarray(y, dtype=np.float64)
+    tol = (K * 2.0 ** -23 + (q + 1) * 2.0 ** -11) * A if tensor_path else K * 2.0 ** -24 * A
+    if out_f16:
+        tol = tol + 2.0 ** -11 * np.abs(ref) * 1.001 + 2.0 ** -24      # (+ fp16 subnormal spacing)
+    bad = np.abs(y64 - ref) > tol
+    if bad.any():
+        i = np.argwhere(bad)[0]
+        raise AssertionError(f"{where}: {int(bad.sum())} of {bad.size} elements outside the bound, first at {tuple(i)}: "
+                             f"got {y64[tuple(i)]!r}, want {ref[tuple(i)]!r}, tolerance {tol[tuple(i)]!r}")

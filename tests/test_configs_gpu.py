@@ -1,7 +1,8 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (C-ABI calls on a
-stream, library-owned scratch): every shape of configs 0, 1 and 3 at M = 1, and the small-batch sweep's
-extremes on one 8B shape, and four calls of the prefill configuration.  The 8B shapes at M = 1 are compared in full against the fp64 oracle; the 70B shapes on
-a seeded sample of output rows (first and last tiles plus random rows), which the oracle computes row by row.
+"""Parity at the benchmark's full sizes, in the launch configurations bench.py times (C-ABI calls on a stream with
+library-owned scratch, and the chained decode entry): every call of configs 0, 1, 2, 3 and 4a, and two layers of the
+32-layer stack of config 4b with their own seeds.  The 8B shapes at M = 1 are compared in full against the fp64
+oracle; the larger problems on a seeded sample of output rows (first and last tiles plus random rows) x all tokens,
+which the oracle computes row by row.  Every comparison is a relative Frobenius error AND an element-wise bound.
 """
 
 import numpy as np
@@ -15,7 +16,7 @@ from workloads import synth
 
 pytestmark = pytest.mark.gpu
 
-from gpu_util import gemm_f16, pack_layer  # noqa: E402
+from gpu_util import assert_elementwise, gemm_f16, pack_layer, x_dev  # noqa: E402
 
 TOL_F16 = 1e-3
 
@@ -44,43 +45,108 @@ def test_config0_single_gemv():
     assert hlq.rel_fro_error(y, ref) <= TOL_F16
 
 
-@pytest.mark.parametrize("call", [c for c in workloads.config3_calls() if c.q == 2 or c.name in ("o", "down")],
-                         ids=lambda c: f"{c.name}-q{c.q}")
+def _sample_rows(N, n_random, seed):
+    rng = np.random.default_rng(seed)
+    return np.unique(np.concatenate([np.arange(min(32, N)), np.arange(max(0, N - 32), N), rng.integers(0, N, n_random)]))
+
+
+@pytest.mark.parametrize("call", workloads.config3_calls(), ids=lambda c: f"{c.name}-q{c.q}")
 def test_config3_shapes_sampled_rows(call):
     layer, X, y = _run(call)
-    rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([np.arange(32), np.arange(call.N - 32, call.N),
-                                     rng.integers(0, call.N, 1024)]))
+    rows = _sample_rows(call.N, 1024, 5)
     ref = hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
     assert np.all(np.isfinite(y))
     assert hlq.rel_fro_error(y[:, rows], ref) <= TOL_F16
+    A = hlq.magnitude_bound(X, layer.scales[rows], layer.offsets[rows], call.G)
+    assert_elementwise(y[:, rows], ref, A, call.q, call.K, False, True, f"config 3 {call.name} q{call.q}")
 
 
-@pytest.mark.parametrize("M", [2, 32])
-def test_config2_small_batch_extremes_on_gate_up(M):
-    call = [c for c in workloads.config2_calls() if c.name == "gate_up" and c.q == 2 and c.M == M][0]
-    layer, X, y = _run(call)
-    rng = np.random.default_rng(6)
-    rows = np.unique(np.concatenate([np.arange(16), np.arange(call.N - 16, call.N), rng.integers(0, call.N, 2048)]))
-    ref = hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
-    assert hlq.rel_fro_error(y[:, rows], ref) <= TOL_F16
+_CFG2 = workloads.config2_calls()
 
 
-@pytest.mark.parametrize("name,M", [("gate_up", 2048), ("down", 2048), ("qkv", 512), ("o", 128)])
-def test_config4_prefill_shapes_sampled(name, M):
-    """The prefill configuration at full size (tensor-core path; CTA pairs for M = 512 and 2048, whole rounds plus
-    the K-split tail stripe on gate_up): sampled weight rows x sampled tokens against the oracle."""
-    call = [c for c in workloads.config4_prefill_calls() if c.name == name and c.M == M][0]
-    layer, X, y = _run(call)
-    rng = np.random.default_rng(7)
-    rows = np.unique(np.concatenate([np.arange(32), np.arange(call.N - 32, call.N), rng.integers(0, call.N, 1024)]))
-    toks = np.unique(np.concatenate([np.arange(8), np.arange(call.M - 8, call.M), rng.integers(0, call.M, 112)]))
-    ref = hlq.matmul(X[toks], layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
-    got = y[np.ix_(toks, rows)]
-    assert np.all(np.isfinite(y))
-    assert hlq.rel_fro_error(got, ref) <= TOL_F16
-    assert max(hlq.rel_fro_error(got[i], ref[i]) for i in range(len(toks))) <= 2 * TOL_F16
+@pytest.mark.parametrize("name,q", sorted({(c.name, c.q) for c in _CFG2}))
+def test_config2_every_call_of_the_small_batch_sweep(name, q):
+    """All six batch sizes of the sweep on one (layer, q): sampled weight rows x all tokens, norm and element-wise."""
+    calls = [c for c in _CFG2 if c.name == name and c.q == q]
+    c0 = calls[0]
+    layer = workloads.hlq_layer(0, c0.tag, c0.q, c0.G, c0.N, c0.K)
+    packed = pack_layer(layer)
+    rows = _sample_rows(c0.N, 1024, 6)
+    for call in calls:
+        X = synth.activations(0, call.tag + f"/x{call.M}", call.M, call.K, outliers=True)
+        y = gemm_f16(X, packed, call.N, call.K)
+        ref = hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
+        assert np.all(np.isfinite(y))
+        assert hlq.rel_fro_error(y[:, rows], ref) <= TOL_F16, call
+        A = hlq.magnitude_bound(X, layer.scales[rows], layer.offsets[rows], call.G)
+        assert_elementwise(y[:, rows], ref, A, call.q, call.K, call.M >= 9, True, f"config 2 {name} q{q} M{call.M}")
     assert elutq.elutq_device_status() == 0
+
+
+@pytest.mark.parametrize("name", ["qkv", "o", "gate_up", "down"])
+def test_config4_every_prefill_call(name):
+    """The prefill configuration at full size (tensor-core path; CTA pairs for M = 512 and 2048, whole rounds plus
+    the K-split tail stripe on gate_up): sampled weight rows x all tokens against the oracle, norm and element-wise."""
+    calls = [c for c in workloads.config4_prefill_calls() if c.name == name]
+    c0 = calls[0]
+    layer = workloads.hlq_layer(0, c0.tag, c0.q, c0.G, c0.N, c0.K)
+    packed = pack_layer(layer)
+    rows = _sample_rows(c0.N, 512, 7)
+    for call in calls:
+        X = synth.activations(0, call.tag + f"/x{call.M}", call.M, call.K)
+        y = gemm_f16(X, packed, call.N, call.K)
+        ref = hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], call.G)
+        got = y[:, rows]
+        assert np.all(np.isfinite(y))
+        assert hlq.rel_fro_error(got, ref) <= TOL_F16, call
+        assert max(hlq.rel_fro_error(got[i], ref[i]) for i in range(call.M)) <= 2 * TOL_F16, call
+        A = hlq.magnitude_bound(X, layer.scales[rows], layer.offsets[rows], call.G)
+        assert_elementwise(got, ref, A, call.q, call.K, True, True, f"config 4a {name} M{call.M}")
+    assert elutq.elutq_device_status() == 0
+
+
+@pytest.mark.parametrize("layer_index", [0, 17])
+def test_config4_stack_layers_with_their_own_seeds(layer_index):
+    """Two layers of the 32-layer stack (four linears each, their own seeds), as separate calls and as one chain."""
+    calls = [c for c in workloads.config4_stack_calls() if c.name.startswith(f"L{layer_index}.")]
+    assert len(calls) == 4
+    layers = [workloads.hlq_layer(0, c.tag, c.q, c.G, c.N, c.K) for c in calls]
+    packed = [pack_layer(l) for l in layers]
+    Xs = [synth.activations(0, c.tag + "/x", 1, c.K) for c in calls]
+    xd = [x_dev(x) for x in Xs]
+    Yc = [torch.zeros((1, c.N), dtype=torch.float16, device="cuda") for c in calls]
+    plan = elutq.elutq_chain_plan([(xd[i], packed[i], Yc[i], c.N, c.K) for i, c in enumerate(calls)])
+    elutq.elutq_chain_run(plan, 4)
+    assert elutq.elutq_chain_status(plan) == 0
+    for i, c in enumerate(calls):
+        ref = hlq.matmul(Xs[i], layers[i].planes, layers[i].scales, layers[i].offsets, c.G)
+        A = hlq.magnitude_bound(Xs[i], layers[i].scales, layers[i].offsets, c.G)
+        ys = gemm_f16(Xs[i], packed[i], c.N, c.K)
+        for y, how in ((ys, "separate call"), (Yc[i].cpu().numpy(), "chain")):
+            assert hlq.rel_fro_error(y, ref) <= TOL_F16, (c.name, how)
+            assert_elementwise(y, ref, A, c.q, c.K, False, True, f"{c.name} {how}")
+    elutq.elutq_chain_forget(plan)
+
+
+@pytest.mark.parametrize("q", [2, 3, 4])
+def test_config1_step_through_the_chain_entry(q):
+    """The benchmark's launch configuration: the four linears of one bit-width as one chain, compared in full."""
+    calls = [c for c in workloads.config1_calls() if c.q == q]
+    layers = [workloads.hlq_layer(0, c.tag, c.q, c.G, c.N, c.K) for c in calls]
+    packed = [pack_layer(l) for l in layers]
+    Xs = [synth.activations(0, c.tag + "/x", 1, c.K) for c in calls]
+    xd = [x_dev(x) for x in Xs]
+    Y = [torch.zeros((1, c.N), dtype=torch.float16, device="cuda") for c in calls]
+    plan = elutq.elutq_chain_plan([(xd[i], packed[i], Y[i], c.N, c.K) for i, c in enumerate(calls)])
+    for _ in range(3):
+        elutq.elutq_chain_run(plan, len(calls))
+    assert elutq.elutq_chain_status(plan) == 0
+    for i, c in enumerate(calls):
+        ref = hlq.matmul(Xs[i], layers[i].planes, layers[i].scales, layers[i].offsets, c.G)
+        y = Y[i].cpu().numpy()
+        assert hlq.rel_fro_error(y, ref) <= TOL_F16, c
+        assert_elementwise(y, ref, hlq.magnitude_bound(Xs[i], layers[i].scales, layers[i].offsets, c.G), c.q, c.K, False, True, c.name)
+    elutq.elutq_chain_forget(plan)
 
 
 def test_smoke_entry_runs():

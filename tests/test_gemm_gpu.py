@@ -11,7 +11,7 @@ from workloads import synth
 
 pytestmark = pytest.mark.gpu
 
-from gpu_util import gemm_f16, gemm_f32, pack_layer, x_dev  # noqa: E402
+from gpu_util import assert_elementwise, gemm_f16, gemm_f32, pack_layer, x_dev  # noqa: E402
 
 TOL_F32 = 5e-6
 TOL_F16 = 1e-3
@@ -33,8 +33,11 @@ def test_batched_gemm_matches_oracle(q, G, N, K, M):
     assert hlq.rel_fro_error(y32, ref) <= TOL_F32
     for m in range(M):                                   # every activation row on its own, too
         assert hlq.rel_fro_error(y32[m], ref[m]) <= 2 * TOL_F32
+    A = hlq.magnitude_bound(X, layer.scales, layer.offsets, G)
+    assert_elementwise(y32, ref, A, q, K, False, False, "batched look-up kernel, fp32 out")
     y16 = gemm_f16(X, packed, N, K)                                # default path
     assert hlq.rel_fro_error(y16, ref) <= TOL_F16
+    assert_elementwise(y16, ref, A, q, K, M >= 9 and G == 128, True, "default path, fp16 out")
     if M < 9 or G != 128:                                # below the tensor-core threshold: the same kernels
         assert np.array_equal(y16.view(np.uint16), y32.astype(np.float16).view(np.uint16))
 
@@ -78,10 +81,13 @@ def test_prefill_sized_batch_on_a_layer_sized_matrix():
     X = synth.activations(23, "prefill/x", M, K)
     packed = pack_layer(layer)
     ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    A = hlq.magnitude_bound(X, layer.scales, layer.offsets, G)
     y16 = gemm_f16(X, packed, N, K)                                  # default path for M >= 9: tensor cores
     assert hlq.rel_fro_error(y16, ref) <= TOL_F16
+    assert_elementwise(y16, ref, A, q, K, True, True, "tensor-core path, fp16 out")
     y32 = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)           # look-up-table kernels
     assert hlq.rel_fro_error(y32, ref) <= TOL_F32
+    assert_elementwise(y32, ref, A, q, K, False, False, "look-up kernels, fp32 out")
 
 
 def test_workspace_entry_and_reproducibility_for_batches():

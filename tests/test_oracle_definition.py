@@ -166,3 +166,29 @@ def test_fp16_rounding_and_error_metric():
     assert h.dtype == np.float16 and float(h[0, 0]) == 1.0 and float(h[0, 1]) == 65504.0
     assert hlq.rel_fro_error(np.array([3.0, 4.0]), np.array([3.0, 4.0])) == 0.0
     assert hlq.rel_fro_error(np.array([0.0, 0.0]), np.array([3.0, 4.0])) == pytest.approx(1.0)
+
+
+def test_magnitude_bound_dominates_the_product_of_magnitudes_for_any_planes():
+    # pin of oracle.hlq.magnitude_bound (the scale of the element-wise parity bounds): for random signed
+    # parameters and ALL bit patterns of a tiny group, and for random planes of a larger layer, it is at least
+    # |X| |W_hat|^T, and it is attained when every weight of a group sits at the group's extreme value
+    rng = np.random.default_rng(11)
+    q, G, N, K = 2, 2, 1, 4
+    s = rng.normal(0, 0.02, (N, K // G, q)).astype(np.float16)
+    z = rng.normal(0, 0.01, (N, K // G)).astype(np.float16)
+    X = rng.normal(0, 1, (2, K)).astype(np.float16)
+    A = hlq.magnitude_bound(X, s, z, G)
+    worst = np.zeros_like(A)
+    for code in range(1 << (q * N * K)):
+        bits = np.array([(code >> i) & 1 for i in range(q * N * K)], dtype=np.uint8).reshape(q, N, K)
+        W = hlq.reconstruct(bits, s, z, G)
+        worst = np.maximum(worst, np.abs(np.asarray(X, dtype=np.float64)) @ np.abs(W).T)
+    assert np.all(A >= worst - 1e-15)
+    assert np.allclose(A, worst, rtol=1e-12)          # the maximum over all planes attains the bound
+    q, G, N, K = 3, 32, 40, 256
+    s = rng.normal(0, 0.02, (N, K // G, q)).astype(np.float16)
+    z = rng.normal(0, 0.01, (N, K // G)).astype(np.float16)
+    X = rng.normal(0, 1, (5, K)).astype(np.float16)
+    planes = rng.integers(0, 2, (q, N, K)).astype(np.uint8)
+    W = hlq.reconstruct(planes, s, z, G)
+    assert np.all(hlq.magnitude_bound(X, s, z, G) >= np.abs(np.asarray(X, dtype=np.float64)) @ np.abs(W).T - 1e-12)

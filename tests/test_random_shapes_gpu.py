@@ -10,7 +10,7 @@ from workloads import synth
 
 pytestmark = pytest.mark.gpu
 
-from gpu_util import gemm_f16, gemm_f32, pack_layer  # noqa: E402
+from gpu_util import assert_elementwise, gemm_f16, gemm_f32, pack_layer  # noqa: E402
 
 
 def _cases():
@@ -36,11 +36,15 @@ def test_random_shape(i, q, G, N, K, M):
     y32 = gemm_f32(X, packed, N, K)
     assert np.all(np.isfinite(y32))
     assert hlq.rel_fro_error(y32, ref) <= (1e-3 if tensor_path else 5e-6)
+    A = hlq.magnitude_bound(X, layer.scales, layer.offsets, G)
+    assert_elementwise(y32, ref, A, q, K, tensor_path, False, "default path, fp32 out")
     y16 = gemm_f16(X, packed, N, K)
     assert hlq.rel_fro_error(y16, ref) <= 1e-3
+    assert_elementwise(y16, ref, A, q, K, tensor_path, True, "default path, fp16 out")
     if tensor_path:
         ylut = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)
         assert hlq.rel_fro_error(ylut, ref) <= 5e-6
+        assert_elementwise(ylut, ref, A, q, K, False, False, "look-up kernels, fp32 out")
     assert elutq.elutq_device_status() == 0
 
 
@@ -68,6 +72,7 @@ def test_random_prefill_shape(i, q, N, K, M):
     y16 = gemm_f16(X, packed, N, K)
     assert np.all(np.isfinite(y16))
     assert hlq.rel_fro_error(y16, ref) <= 1e-3
-    rows = range(0, M, max(1, M // 32))
-    assert max(hlq.rel_fro_error(y16[m], ref[m]) for m in rows) <= 2e-3
+    assert max(hlq.rel_fro_error(y16[m], ref[m]) for m in range(M)) <= 2e-3
+    assert_elementwise(y16, ref, hlq.magnitude_bound(X, layer.scales, layer.offsets, G), q, K, True, True,
+                       "tensor-core path, fp16 out")
     assert elutq.elutq_device_status() == 0
