@@ -335,6 +335,17 @@ int elutq_hlq_fit(const void* W, int q, int G, int N, int K, int t_max, uint8_t*
  */
 int elutq_device_status(void* stream, int* status);
 
+/*
+ * Test entry for the bounded waits of the tensor-core kernel (9 <= M <= 128, G = 128, K >= 384): the call is
+ * launched with the issuing thread told to issue no MMA and no completion signal and with the poll limit of the
+ * device-side waits set to `wait_limit`, so that the waits for MMA completion run out: the kernel gives up
+ * waiting, still joins every barrier, frees its tensor memory and returns; elutq_device_status then reads
+ * ELUTQ_DEVICE_WAIT_EXPIRED.  Y (float [M][N]) receives undefined values.  Nothing faults and nothing waits
+ * without a limit.  Call elutq_release_scratch afterwards to clear the status.
+ */
+int elutq_test_wait_expiry(const void* X, const void* packed, float* Y, int M, int N, int K,
+                           unsigned wait_limit, void* stream);
+
 /* Number of kernel launches the library has issued in this process (all entry
  * points); lets a benchmark count its launches. */
 unsigned long long elutq_launch_count(void);

@@ -64,6 +64,7 @@ _SIGNATURES = {
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
+    "elutq_test_wait_expiry": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p]),
     "elutq_reserve": (c_int, [c_int, c_int, c_int, c_void_p]),
     "elutq_scratch_address": (c_int, [c_void_p, c_int, ctypes.POINTER(c_void_p), ctypes.POINTER(c_size_t)]),
 }
@@ -266,3 +267,8 @@ def elutq_scratch_address(kind: int, stream=None):
     ptr, nb = c_void_p(0), c_size_t(0)
     _check(lib().elutq_scratch_address(_stream(stream), kind, ctypes.byref(ptr), ctypes.byref(nb)), "elutq_scratch_address")
     return ptr.value, nb.value
+
+
+def elutq_test_wait_expiry(X, packed, Y, M: int, N: int, K: int, wait_limit: int, stream=None) -> None:
+    _check(lib().elutq_test_wait_expiry(_ptr(X), _ptr(packed), _ptr(Y), M, N, K, wait_limit, _stream(stream)),
+           "elutq_test_wait_expiry")

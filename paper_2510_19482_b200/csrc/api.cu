@@ -16,6 +16,8 @@ namespace elutq {
 namespace {
 
 thread_local int g_last_cuda_error = 0;
+thread_local unsigned g_test_flags = 0;        // set around one call by elutq_test_wait_expiry
+thread_local unsigned g_test_wait_limit = 0;
 std::atomic<unsigned long long> g_launches{0};
 
 struct BlobMeta { int q, G, N, K; };
@@ -201,7 +203,9 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     a.partials = reinterpret_cast<float*>(partials);
     a.M = M; a.N = N; a.K = K;
     a.n_rb = g.n_rb; a.n_kc = g.n_kc;
-    a.flags = flags;
+    a.flags = flags | g_test_flags;
+    a.wait_limit = g_test_wait_limit;
+    a.items_q = 0; a.items_r = 0; a.active_warps = 0; a.ranges = 0; a.rb_q = 0; a.rb_r = 0; a.cpc = 1; a.cluster_reduce = 0;
     const int sms = num_sms();
     int ce;
     const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY |
@@ -370,6 +374,17 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host, in
     e = cudaMemcpyAsync(Y_host, yd, yb, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e);
     return ELUTQ_OK;
+}
+
+int elutq_test_wait_expiry(const void* X, const void* packed, float* Y, int M, int N, int K, unsigned wait_limit, void* stream) {
+    if (M < ELUTQ_TENSOR_MIN_M || M > 128 || wait_limit == 0) return ELUTQ_ERR_UNSUPPORTED;   // the one-token-tile schedule only
+    if (K < 3 * 128) return ELUTQ_ERR_UNSUPPORTED;                                           // a wait needs a third K step
+    g_test_flags = kFlagTestNoMma;
+    g_test_wait_limit = wait_limit;
+    const int st = run_gemm(X, packed, Y, M, N, K, ELUTQ_FLAG_OUT_F32, nullptr, 0, true, stream);
+    g_test_flags = 0;
+    g_test_wait_limit = 0;
+    return st;
 }
 
 int elutq_device_status(void* stream, int* status) {

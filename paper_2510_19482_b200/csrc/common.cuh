@@ -64,6 +64,7 @@ struct GemmArgs {
     int cpc;                 // chunks per CTA in the aligned partition
     int cluster_reduce;      // 1: launched as clusters of n_kc CTAs (one per chunk, same row range): partials stay in
                              //    shared memory and are reduced through distributed shared memory
+    unsigned wait_limit;     // poll limit of the tensor-core kernel's bounded waits (0: the default)
 };
 
 // Kernel launchers (defined in the .cu files); return a cudaError_t value.
@@ -158,7 +159,10 @@ __device__ __forceinline__ float ld_cluster_f32(const float* local_smem_ptr, uns
 }
 // Device status codes (word 0 of the control area; read back by elutq_device_status / elutq_chain_status).
 constexpr unsigned kStatusWaitExpired = 0x7C05u;    // a bounded wait ran out
-constexpr unsigned kStatusBlobMismatch = 0x7C0Bu;   // the blob header does not describe what the kernel was launched for
+constexpr unsigned kStatusBlobMismatch = 0x7C0Bu;
+// Internal flag (never accepted from callers; set by elutq_test_wait_expiry only): the tensor-core kernel's issuing
+// thread issues no MMA and no commit, so that the other threads' bounded waits for MMA completion run out.
+constexpr unsigned kFlagTestNoMma = 0x20000000u;   // the blob header does not describe what the kernel was launched for
 
 // Every GEMM kernel compares the header of the blob it was handed with the geometry it was launched for before it
 // reads any tile: a stale description of an address that now holds another blob must never turn into reads

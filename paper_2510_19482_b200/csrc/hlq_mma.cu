@@ -66,8 +66,8 @@ __device__ __forceinline__ uint64_t desc_swizzle128(uint32_t saddr) {
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -279,9 +279,10 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
     // One thread's view of a completion barrier: every thread polls for itself; a thread whose wait runs out
     // raises the status word once and stops waiting, but keeps taking part in every CTA-wide barrier.
     bool ok = true;
+    const uint32_t wait_limit = a.wait_limit ? a.wait_limit : kWaitLimit;
     auto wait_mma = [&](int which, uint32_t parity) {
         if (!ok) return;
-        if (!mbar_wait(bar_addr + 8u * which, parity)) {
+        if (!mbar_wait(bar_addr + 8u * which, parity, wait_limit)) {
             ok = false;
             if (a.counters != nullptr) atomicExch(a.counters, 0x7C05u);
         }
@@ -293,7 +294,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         if (!ok) return;
         bool done = false;
         if constexpr (CG == 2) {
-            for (uint32_t i = 0; i < kWaitLimit && !done; ++i) {
+            for (uint32_t i = 0; i < wait_limit && !done; ++i) {
                 uint32_t r;
                 asm volatile("{\n\t.reg .pred p;\n\t"
                              "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
@@ -302,7 +303,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
                 done = r != 0;
             }
         } else {
-            done = mbar_wait(bar_addr + 8u * which, parity);
+            done = mbar_wait(bar_addr + 8u * which, parity, wait_limit);
         }
         if (!done) {
             ok = false;
@@ -411,6 +412,7 @@ __global__ void __launch_bounds__(kMmaThreads + (WS ? 32 : 0), 1) hlq_mma_kernel
         // activation stages, so the copy for step s + 1 never waits for the MMAs of step s - 1 either.
         auto issue_step = [&](int step, int stage, int wt) {
             if (tid != 0) return;
+            if (a.flags & kFlagTestNoMma) return;      // test only: nothing is issued, nothing completes, the waits run out
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int kk = 0; kk < kStepK / 16; ++kk) {

@@ -79,7 +79,7 @@ extern "C" int elutq_lut_gemm_static(const void* X, const void* packed, void* Y,
     a.n_rb = (int)n_rb; a.n_kc = (int)n_kc;
     a.flags = 0u;
     a.items_q = 0; a.items_r = 0; a.active_warps = 0;
-    a.ranges = 0; a.rb_q = 0; a.rb_r = 0; a.cpc = 1; a.cluster_reduce = 0;
+    a.ranges = 0; a.rb_q = 0; a.rb_r = 0; a.cpc = 1; a.cluster_reduce = 0; a.wait_limit = 0;
     const int sms = device_sm_count();
     const int ce = (M == 1) ? launch_lut_gemv(a, q, G, sms, (cudaStream_t)stream)
                             : launch_lut_gemm(a, q, G, sms, (cudaStream_t)stream);

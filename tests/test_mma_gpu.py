@@ -89,3 +89,23 @@ def test_tensor_core_path_is_bit_reproducible(q, N, K, M):
         b = gemm_f16(X, packed, N, K)
         assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
     assert elutq.elutq_device_status() == 0
+
+
+def test_a_wait_for_mma_completion_that_runs_out_is_reported_and_the_stream_stays_usable():
+    # The test entry launches the one-token-tile kernel with its issuing thread told to issue nothing and the poll
+    # limit at 4096: every thread's wait for the MMAs of two steps ago runs out, the kernel stops waiting, joins its
+    # barriers, frees its tensor memory and returns; the status word says so.  The next ordinary call on the same
+    # stream is correct.
+    q, G, N, K, M = 2, 128, 512, 2048, 64
+    layer = workloads.hlq_layer(33, "mma/expiry", q, G, N, K)
+    X = synth.activations(33, "mma/expiry/x", M, K)
+    packed = pack_layer(layer)
+    elutq.elutq_release_scratch()
+    Y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    elutq.elutq_test_wait_expiry(x_dev(X), packed, Y, M, N, K, 4096)
+    assert elutq.elutq_device_status() == 0x7C05
+    elutq.elutq_release_scratch()
+    ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
+    y = gemm_f32(X, packed, N, K)
+    assert elutq.elutq_device_status() == 0
+    assert hlq.rel_fro_error(y, ref) <= TOL
