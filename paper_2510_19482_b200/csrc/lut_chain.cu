@@ -409,7 +409,8 @@ __device__ __forceinline__ void lookup_calls(const ChainCtx& x) {
             mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
             if (b == 0) chain_items<Q, G, 0>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
             else chain_items<Q, G, 1>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
-            mbar_arrive(bar_free(b));         // this thread no longer reads buffer b
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_free(b));   // this warp no longer reads buffer b
             seg_vp += (size_t)d->n_rb * C::TILE_BYTES;
         }
         if (d->n_kc == 1) {
@@ -461,10 +462,12 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
     if (tid == 0) {
         sh->abort = 0;
         sh->epoch = ctl->epoch;
-        mbar_init(bar_full(0), kBuilderThreads);
-        mbar_init(bar_full(1), kBuilderThreads);
-        mbar_init(bar_free(0), kLookupWarps * 32);
-        mbar_init(bar_free(1), kLookupWarps * 32);
+        // one arrival per warp (its lane 0, after the warp has converged): 32 arrivals of a warp on one barrier word
+        // would be 32 serialised shared-memory atomics
+        mbar_init(bar_full(0), kBuilderWarps);
+        mbar_init(bar_full(1), kBuilderWarps);
+        mbar_init(bar_free(0), kLookupWarps);
+        mbar_init(bar_free(1), kLookupWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     cp_async_wait_all();
@@ -531,7 +534,8 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
                             raise_abort(status);
                         bar_builders();
                     }
-                    mbar_arrive(bar_full(b));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_full(b));
                 }
             }
             if (bt < 9) cp_async_wait_all();
