@@ -51,8 +51,10 @@ constexpr int kOffBar = kOffGsum + 128;
 constexpr int kOffShared = kOffBar + 32;
 constexpr int kSlotBytes = 144;                           // descriptor (128) + this CTA's share of the call (16)
 constexpr int kOffDesc = kOffGsum + 256;                  // builders' descriptor ring
-constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // look-up and finisher warps: a descriptor ring per warp
-constexpr int kChainSmem = kOffWarpDesc + (kLookupWarps + kFinisherWarps) * kDescSlots * kSlotBytes;
+constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // finisher warps: a descriptor ring per warp
+constexpr int kOffJobRec = kOffWarpDesc + kFinisherWarps * kDescSlots * kSlotBytes;   // job records, written by the builders
+constexpr int kJobRecs = 4;
+constexpr int kChainSmem = kOffJobRec + kJobRecs * 64;
 constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
 constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
 
@@ -129,9 +131,30 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, unsigned parity) {
 struct ChainShared {
     volatile int abort;                       // a wait ran out: stop waiting
     unsigned epoch;
+    volatile unsigned recs_published;         // job records written so far (by the builders)
 };
 
+// What the look-up warps need to know of one table job (a call's K chunk on this CTA), written by the builders
+// before they build the job's tables: the look-up warps follow these records and never touch a descriptor.
+struct JobRec {
+    const uint8_t* tile0;                     // the job's first item (row block rb0 of chunk kc)
+    unsigned long long* out;                  // tagged partial sums of chunk kc (row 0), or nullptr: no K split, store Y
+    void* Y;
+    unsigned* done;                           // completion counter of the call (used without a K split)
+    int rb0, rb1, N;
+    unsigned flags, tag;
+    int last;                                 // 1: the call's last job on this CTA
+    int stop;                                 // 1: no more jobs in this launch
+    int pad[1];
+};
+static_assert(sizeof(JobRec) == 64, "job record size");
+
+
 extern __shared__ __align__(1024) uint8_t chain_smem[];
+
+__device__ __forceinline__ JobRec* job_rec(unsigned job) {
+    return reinterpret_cast<JobRec*>(chain_smem + kOffJobRec) + (job & (kJobRecs - 1));
+}
 
 __device__ __forceinline__ ChainShared* chain_shared() { return reinterpret_cast<ChainShared*>(chain_smem + kOffShared); }
 struct ChainSlot {                            // what a role keeps of a call in shared memory
@@ -143,8 +166,8 @@ __device__ __forceinline__ ChainSlot* chain_slot(int c) {
     return reinterpret_cast<ChainSlot*>(chain_smem + kOffDesc) + (c & (kDescSlots - 1));
 }
 __device__ __forceinline__ ChainCall* chain_desc(int c) { return &chain_slot(c)->d; }
-__device__ __forceinline__ ChainSlot* warp_slot(int lw, int c) {
-    return reinterpret_cast<ChainSlot*>(chain_smem + kOffWarpDesc) + lw * kDescSlots + (c & (kDescSlots - 1));
+__device__ __forceinline__ ChainSlot* warp_slot(int fw, int c) {
+    return reinterpret_cast<ChainSlot*>(chain_smem + kOffWarpDesc) + fw * kDescSlots + (c & (kDescSlots - 1));
 }
 // Copies descriptor c and this CTA's share of call c into a slot: nine 16-byte pieces, one per lane.
 __device__ __forceinline__ void slot_fetch(ChainSlot* dst, const ChainCall* calls, const int4* parts, int grid, int c, int piece) {
@@ -300,35 +323,33 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
     }
 }
 
-// Items of one chunk (kc) of call d on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of
-// the chunk on entry and, on exit, the item at after_vp (its first item of the CTA's next chunk or of the next
-// call; nullptr: none).
+// Items of one job on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of the job on entry
+// and, on exit, the item at after_vp (its first item of the next job; nullptr: none).
 template <int Q, int G, int B>
-__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const ChainCall* d, const int rb0,
-                                            const int rb1, const int kc, const uint8_t* after_vp, const uint8_t* seg_vp,
-                                            const unsigned tag, const int lw, const int lane) {
+__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const JobRec* r, const uint8_t* vp,
+                                            const uint8_t* after_vp, const int lw, const int lane) {
     using C = Cfg<Q, G>;
     const uint8_t* const tab = chain_smem + B * kTableBytes;
     const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
     const int h = lane >> 4, l = lane & 15;
     float S[C::GL];
     load_group_sums<G>(S, gsum, h, l, true);
-    const int n_rb = d->n_rb;
-    const uint8_t* vp = seg_vp;
-    unsigned long long* out = d->slots + (size_t)kc * ((size_t)n_rb * kTileRows) + l;
-    for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
-        // next item of this warp: the same chunk, else the one the caller names
-        const bool in_seg = rb + kLookupWarps < rb1;
-        const uint8_t* nvp = in_seg ? vp + kLookupWarps * C::TILE_BYTES : after_vp;
+    const int rb1 = r->rb1;
+    unsigned long long* out = r->out;
+    const unsigned long long tag_hi = (unsigned long long)r->tag << 32;
+    for (int rb = r->rb0 + lw; rb < rb1; rb += kLookupWarps) {
+        // next item of this warp: the same job, else the one the caller names
+        const bool in_job = rb + kLookupWarps < rb1;
+        const uint8_t* nvp = in_job ? vp + kLookupWarps * C::TILE_BYTES : after_vp;
         const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
         float y;
-        if (in_seg || after_vp != nullptr) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
+        if (in_job || after_vp != nullptr) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
         else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
         if (h == 0) {
-            if (d->n_kc == 1) {
-                if (rb * kTileRows + l < d->N) chain_store(d->Y, d->flags, (size_t)(rb * kTileRows + l), y);
+            if (out == nullptr) {
+                if (rb * kTileRows + l < r->N) chain_store(r->Y, r->flags, (size_t)(rb * kTileRows + l), y);
             } else {
-                st_relaxed_u64(out + rb * kTileRows, ((unsigned long long)tag << 32) | __float_as_uint(y));
+                st_relaxed_u64(out + rb * kTileRows + l, tag_hi | __float_as_uint(y));
             }
         }
         vp = nvp;
@@ -365,60 +386,50 @@ __device__ __forceinline__ const ChainSlot* desc_next(const ChainCtx& x, int slo
     return warp_slot(slot_warp, c);
 }
 
-// Look-up role of one warp over the calls of a launch.  (A launch covers calls of one (q, G): a variant that switched
-// between per-q instances of this function inside one kernel was measured three times slower, whether the instances
-// were inlined or called.)
+// Look-up role of one warp: it follows the job records the builders publish.  (A launch covers calls of one (q, G):
+// a variant that switched between per-q instances of this function inside one kernel was measured three times slower,
+// whether the instances were inlined or called.)
 template <int Q, int G>
-__device__ __forceinline__ void lookup_calls(const ChainCtx& x) {
+__device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
     using C = Cfg<Q, G>;
-    const int lane = threadIdx.x & 31, lw = threadIdx.x >> 5, bid = blockIdx.x;
+    const int lane = threadIdx.x & 31, lw = threadIdx.x >> 5;
     const int h = lane >> 4, l = lane & 15;
+    ChainShared* sh = chain_shared();
     uint32_t colp[4];
     make_colp<G>(colp, h, l);
-    unsigned job = 0;                         // table jobs (call, chunk) of this CTA, counted alike by every role
     Item<Q, G> buf;
-    bool carried = false;                     // buf already holds this warp's first item of the call
-    desc_begin(x, lw, lane);
-    for (int c = x.c_begin; c < x.c_end; ++c) {
-        const ChainSlot* sl = desc_next(x, lw, c, lane);
-        const ChainCall* d = &sl->d;
-        if (bid >= d->n_ctas) continue;
-        const ChainPart p = chain_part(sl);
-        const unsigned tag = x.epoch * (unsigned)x.n_calls + (unsigned)c + 1u;
-        const uint8_t* seg_vp = d->tiles + ((size_t)p.kc0 * d->n_rb + p.rb0 + lw) * C::TILE_BYTES + lane * 16;
-        const bool items = p.rb0 + lw < p.rb1;
-        if (items && !carried) load_item<Q, G>(buf, seg_vp, seg_vp + (C::PLANE_BYTES - lane * 12), true);
+    bool carried = false;                     // buf already holds this warp's first item of the job
+    const size_t warp_off = (size_t)lw * C::TILE_BYTES + lane * 16;
+    for (unsigned job = 0;; ++job) {
+        const int b = job & 1;
+        mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
+        const JobRec* r = job_rec(job);
+        if (r->stop || sh->abort) break;
+        const bool items = r->rb0 + lw < r->rb1;
+        const uint8_t* vp = r->tile0 + warp_off;
+        if (items && !carried) load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
         carried = false;
-        // what follows this warp's last item of the call: its first item of the next call, when the CTA and the
-        // warp have work there
-        const uint8_t* next_call_vp = nullptr;
-        if (items && c + 1 < x.c_end) {
-            const ChainSlot* sn = warp_slot(lw, c + 1);
-            const ChainCall* dn = &sn->d;
-            if (bid < dn->n_ctas) {
-                const ChainPart pn = chain_part(sn);
-                if (pn.rb0 + lw < pn.rb1) {
-                    next_call_vp = dn->tiles + ((size_t)pn.kc0 * dn->n_rb + pn.rb0 + lw) * C::TILE_BYTES + lane * 16;
-                    carried = true;
-                }
+        // what follows this warp's last item of the job: its first item of the next job, when that job's record is
+        // already there (the builders normally run a job ahead) and the warp has an item in it
+        const uint8_t* after_vp = nullptr;
+        if (items && sh->recs_published > job + 1) {
+            const JobRec* rn = job_rec(job + 1);
+            if (!rn->stop && rn->rb0 + lw < rn->rb1) {
+                after_vp = rn->tile0 + warp_off;
+                carried = true;
             }
         }
-        for (int seg = 0; seg < p.nseg; ++seg, ++job) {
-            const int b = job & 1;
-            const uint8_t* after_vp = seg + 1 < p.nseg ? seg_vp + (size_t)d->n_rb * C::TILE_BYTES : next_call_vp;
-            mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
-            if (b == 0) chain_items<Q, G, 0>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
-            else chain_items<Q, G, 1>(buf, colp, d, p.rb0, p.rb1, p.kc0 + seg, after_vp, seg_vp, tag, lw, lane);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_free(b));   // this warp no longer reads buffer b
-            seg_vp += (size_t)d->n_rb * C::TILE_BYTES;
-        }
-        if (d->n_kc == 1) {
-            __syncwarp();
-            if (lane == 0 && !(d->flags & kCallTestNoSignal)) {
+        if (b == 0) chain_items<Q, G, 0>(buf, colp, r, vp, after_vp, lw, lane);
+        else chain_items<Q, G, 1>(buf, colp, r, vp, after_vp, lw, lane);
+        const bool report = r->out == nullptr && r->last && !(r->flags & kCallTestNoSignal);
+        unsigned* done_c = r->done;
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(bar_free(b));         // this warp no longer reads buffer b (nor the job's record)
+            if (report) {
                 // no K split: this warp stored its rows of Y itself and reports them
                 __threadfence();
-                atomicAdd(x.done + c, 1u);
+                atomicAdd(done_c, 1u);
             }
         }
     }
@@ -461,6 +472,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
     }
     if (tid == 0) {
         sh->abort = 0;
+        sh->recs_published = 0;
         sh->epoch = ctl->epoch;
         // one arrival per warp (its lane 0, after the warp has converged): 32 arrivals of a warp on one barrier word
         // would be 32 serialised shared-memory atomics
@@ -485,7 +497,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
 
     if (warp < kLookupWarps) {
         // ---------------------------------------------------------------- look-up warps
-        lookup_calls<Q, G>(x);
+        lookup_jobs<Q, G>(x);
     } else if (warp < kLookupWarps + kBuilderWarps) {
         // ---------------------------------------------------------------- builder warps
         const int bw = warp - kLookupWarps, bt = tid - kLookupWarps * 32;
@@ -524,6 +536,24 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
                     const int b = job & 1;
                     float2 xv[8];             // requested before the wait for the buffer: the load latency overlaps it
                     load_x_pairs(xv, d->X, p.kc0 + seg, d->K, lane);
+                    if (bt == 0) {
+                        // the job's record, published before the tables are built: the look-up warps may already request
+                        // their first item of this job while they work on the one before (the record's slot was last
+                        // read four jobs ago)
+                        JobRec* r = job_rec(job);
+                        const int kc = p.kc0 + seg;
+                        r->tile0 = d->tiles + ((size_t)kc * d->n_rb + p.rb0) * Cfg<Q, G>::TILE_BYTES;
+                        r->out = d->n_kc > 1 ? d->slots + (size_t)kc * ((size_t)d->n_rb * kTileRows) : nullptr;
+                        r->Y = d->Y;
+                        r->done = done + c;
+                        r->rb0 = p.rb0; r->rb1 = p.rb1; r->N = d->N;
+                        r->flags = d->flags;
+                        r->tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
+                        r->last = seg + 1 == p.nseg;
+                        r->stop = 0;
+                        __threadfence_block();
+                        sh->recs_published = job + 1;
+                    }
                     if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);   // look-ups of job - 2 are over
                     build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), xv, bw, lane);
                     if (seg == 0 && d->guard_call >= 0) {
@@ -541,13 +571,26 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
             if (bt < 9) cp_async_wait_all();
             bar_builders();                   // descriptor c + 3 has landed for every builder thread
         }
+        {   // the record that ends the look-up warps' loop, handed over like a job
+            const int b = job & 1;
+            if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);
+            if (bt == 0) {
+                JobRec* r = job_rec(job);
+                r->rb0 = 0; r->rb1 = 0;
+                r->stop = 1;
+                __threadfence_block();
+                sh->recs_published = job + 1;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full(b));
+        }
     } else {
         // ---------------------------------------------------------------- finisher warps
         // K-split reduction of every call this CTA works on, then the call's completion report
         const int fw = warp - kLookupWarps - kBuilderWarps, ft = tid - (kLookupWarps + kBuilderWarps) * 32;
-        desc_begin(x, kLookupWarps + fw, lane);
+        desc_begin(x, fw, lane);
         for (int c = c_begin; c < c_end; ++c) {
-            const ChainSlot* sl = desc_next(x, kLookupWarps + fw, c, lane);
+            const ChainSlot* sl = desc_next(x, fw, c, lane);
             const ChainCall* d = &sl->d;
             if (bid < d->n_ctas && d->n_kc > 1) {
                 const ChainPart p = chain_part(sl);

@@ -3,8 +3,8 @@
 // Work decomposition
 //   item  = one tile of the packed layout: 16 output rows x 512 input columns (all q planes,
 //           their scales and offsets), processed by one warp.
-//   CTA   = 16 warps; owns a contiguous range of the kc-major item list, so it needs the
-//           activation tables of one K chunk at a time (rebuilt when the range crosses a chunk).
+//   CTA   = 32 warps; owns one K chunk over a row range (aligned partition; a contiguous range of the kc-major item
+//           list where that balances better), so it needs the activation tables of one K chunk at a time.
 //   lane  = 16*h + l: output row l of the tile, super-groups h and h+2 (128 columns each).
 //
 // Tables (step "LUT build"): for every byte-column c of the chunk (8 activations) the 256
@@ -18,8 +18,10 @@
 // multiplies by the group's per-plane scale, adds offset * group activation sum, and the two
 // half-warps are combined with one shuffle.
 //
-// K split: one partial per K chunk goes to the workspace; the warp that arrives last at a row
-// block (arrival counter, wraps to zero) adds the partials in a fixed order and writes Y.
+// K split: one partial sum per K chunk goes to the workspace; a finalize kernel, launched right behind with programmatic
+// dependent launch, adds the chunks in ascending order (bit-reproducible) and writes Y.  ELUTQ_FLAG_CLUSTER_REDUCE keeps
+// the partial sums in shared memory instead and reduces them across a thread-block cluster.  (The chained entry of
+// lut_chain.cu reduces inside its own kernel.)
 #include "lut_core.cuh"
 
 namespace elutq {
