@@ -136,16 +136,18 @@ struct ChainShared {
 
 // What the look-up warps need to know of one table job (a call's K chunk on this CTA), written by the builders
 // before they build the job's tables: the look-up warps follow these records and never touch a descriptor.
-struct JobRec {
+struct JobRec {                               // four 16-byte quarters, each read with one shared-memory load
     const uint8_t* tile0;                     // the job's first item (row block rb0 of chunk kc)
+    int rb0, rb1;                             //   (a record with rb0 == rb1 has no items: the stop record)
     unsigned long long* out;                  // tagged partial sums of chunk kc (row 0), or nullptr: no K split, store Y
     void* Y;
     unsigned* done;                           // completion counter of the call (used without a K split)
-    int rb0, rb1, N;
-    unsigned flags, tag;
+    int N;
+    unsigned flags;
+    unsigned tag;
     int last;                                 // 1: the call's last job on this CTA
     int stop;                                 // 1: no more jobs in this launch
-    int pad[1];
+    int pad;
 };
 static_assert(sizeof(JobRec) == 64, "job record size");
 
@@ -326,18 +328,18 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 // Items of one job on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of the job on entry
 // and, on exit, the item at after_vp (its first item of the next job; nullptr: none).
 template <int Q, int G, int B>
-__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const JobRec* r, const uint8_t* vp,
-                                            const uint8_t* after_vp, const int lw, const int lane) {
+__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
+                                            unsigned long long* out, void* Y, const int N, const unsigned flags,
+                                            const unsigned tag, const uint8_t* vp, const uint8_t* after_vp, const int lw,
+                                            const int lane) {
     using C = Cfg<Q, G>;
     const uint8_t* const tab = chain_smem + B * kTableBytes;
     const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
     const int h = lane >> 4, l = lane & 15;
     float S[C::GL];
     load_group_sums<G>(S, gsum, h, l, true);
-    const int rb1 = r->rb1;
-    unsigned long long* out = r->out;
-    const unsigned long long tag_hi = (unsigned long long)r->tag << 32;
-    for (int rb = r->rb0 + lw; rb < rb1; rb += kLookupWarps) {
+    const unsigned long long tag_hi = (unsigned long long)tag << 32;
+    for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
         // next item of this warp: the same job, else the one the caller names
         const bool in_job = rb + kLookupWarps < rb1;
         const uint8_t* nvp = in_job ? vp + kLookupWarps * C::TILE_BYTES : after_vp;
@@ -347,7 +349,7 @@ __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&co
         else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
         if (h == 0) {
             if (out == nullptr) {
-                if (rb * kTileRows + l < r->N) chain_store(r->Y, r->flags, (size_t)(rb * kTileRows + l), y);
+                if (rb * kTileRows + l < N) chain_store(Y, flags, (size_t)(rb * kTileRows + l), y);
             } else {
                 st_relaxed_u64(out + rb * kTileRows + l, tag_hi | __float_as_uint(y));
             }
@@ -403,26 +405,34 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
     for (unsigned job = 0;; ++job) {
         const int b = job & 1;
         mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
-        const JobRec* r = job_rec(job);
-        if (r->stop || sh->abort) break;
-        const bool items = r->rb0 + lw < r->rb1;
-        const uint8_t* vp = r->tile0 + warp_off;
+        // the job's record in four loads (one round of shared-memory latency instead of a dependent chain of them)
+        const uint4* rq = reinterpret_cast<const uint4*>(job_rec(job));
+        const uint4 q0 = rq[0], q1 = rq[1], q2 = rq[2], q3 = rq[3];
+        if (q3.z != 0u || sh->abort) break;                       // stop record
+        const uint8_t* tile0 = reinterpret_cast<const uint8_t*>(((unsigned long long)q0.y << 32) | q0.x);
+        const int rb0 = (int)q0.z, rb1 = (int)q0.w;
+        unsigned long long* out = reinterpret_cast<unsigned long long*>(((unsigned long long)q1.y << 32) | q1.x);
+        void* Y = reinterpret_cast<void*>(((unsigned long long)q1.w << 32) | q1.z);
+        unsigned* done_c = reinterpret_cast<unsigned*>(((unsigned long long)q2.y << 32) | q2.x);
+        const int N = (int)q2.z;
+        const unsigned flags = q2.w, tag = q3.x;
+        const bool items = rb0 + lw < rb1;
+        const uint8_t* vp = tile0 + warp_off;
         if (items && !carried) load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
         carried = false;
         // what follows this warp's last item of the job: its first item of the next job, when that job's record is
         // already there (the builders normally run a job ahead) and the warp has an item in it
         const uint8_t* after_vp = nullptr;
         if (items && sh->recs_published > job + 1) {
-            const JobRec* rn = job_rec(job + 1);
-            if (!rn->stop && rn->rb0 + lw < rn->rb1) {
-                after_vp = rn->tile0 + warp_off;
+            const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
+            if ((int)n0.z + lw < (int)n0.w) {
+                after_vp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + warp_off;
                 carried = true;
             }
         }
-        if (b == 0) chain_items<Q, G, 0>(buf, colp, r, vp, after_vp, lw, lane);
-        else chain_items<Q, G, 1>(buf, colp, r, vp, after_vp, lw, lane);
-        const bool report = r->out == nullptr && r->last && !(r->flags & kCallTestNoSignal);
-        unsigned* done_c = r->done;
+        if (b == 0) chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, after_vp, lw, lane);
+        else chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, after_vp, lw, lane);
+        const bool report = out == nullptr && q3.y != 0u && !(flags & kCallTestNoSignal);
         __syncwarp();
         if (lane == 0) {
             mbar_arrive(bar_free(b));         // this warp no longer reads buffer b (nor the job's record)
