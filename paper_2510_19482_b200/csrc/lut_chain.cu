@@ -3,25 +3,26 @@
 // A decode step is a fixed sequence of linears on one stream.  Launched one by one, every call pays its own
 // chain of cross-SM hand-overs (kernel start, activation load, table build, K-split reduction, kernel end), during
 // which HBM idles; for the 8B layer shapes that chain is several times longer than the time the call's bytes need.
-// Here one cooperative grid (one 1024-thread CTA per SM) walks a run of consecutive calls that share (q, G) - a
+// Here one grid (one 1024-thread CTA per SM, all resident) walks a run of consecutive calls that share (q, G) - a
 // model has one such pair, so normally the whole list is one launch; a list that mixes them is cut into one
 // launch per run.  Inside a CTA the warps are specialised (Appendix B's two phases run side by side):
 //
 //   * 4 builder warps load the activations of the CTA's next K chunk and fill the other of two table buffers
-//     (fused 8-bit tables, 64 KiB each) while
-//   * 28 look-up warps stream the packed weights of the current chunk (one warp per 16-row x 512-column item,
-//     registers refilled one item ahead, as in lut_gemv.cu) and sum table entries.  Buffers are handed over through
-//     shared-memory mbarriers ("full" / "free" per buffer).
-//   * K-split: every partial sum is stored together with a tag (launch epoch and call number) in one 8-byte
-//     word.  The CTAs that share a row range split its rows among themselves; the builder warps poll (bounded)
-//     the tagged words of their rows, add the chunks in ascending order - bit-reproducible - and write Y.  No
-//     fence, no ticket, no second kernel: the load that finds the tag is the load that brings the value.
+//     (fused 8-bit tables, 64 KiB each); before they build a job they publish a small record of it (first item,
+//     row-block range, where the partial sums go, tag) in shared memory;
+//   * 26 look-up warps follow those records: they stream the packed weights of the job (one warp per 16-row x
+//     512-column item, registers refilled one item ahead as in lut_gemv.cu, also across job boundaries) and sum table
+//     entries.  Buffers are handed over through shared-memory mbarriers ("full" / "free" per buffer, one arrival per
+//     warp, waits suspended in hardware rather than spinning);
+//   * K split: every partial sum is stored together with a tag (launch epoch and call number) in one 8-byte
+//     word.  The CTAs that share a row range split its rows among themselves; 2 finisher warps poll (bounded) the
+//     tagged words of their rows, add the chunks in ascending order - bit-reproducible - and write Y, then report
+//     the call's completion on a counter.  No fence, no ticket, no second kernel for the reduction: the load that
+//     finds the tag is the load that brings the value.
 //   * Ordering: the result is what the calls give when run one after another.  The plan records, from the buffer
 //     addresses, which earlier calls a call really depends on (its X or Y overlaps their Y, or its Y their X);
 //     before the builders read X they wait (bounded) for the completion counters of exactly those calls.  Calls
-//     without such a dependency overlap freely, so HBM keeps streaming across call boundaries.
-//   * The builders also ask L2 for the look-up warps' first items of the next call (cp.async.bulk.prefetch.L2)
-//     a whole call ahead, and a rolling prefetch runs two items ahead of the register loads.
+//     without such a dependency overlap freely, so the weight stream does not stop at call boundaries.
 //
 // Every wait is a bounded poll; when one runs out the CTA raises the plan's status word, stops waiting for
 // the rest of the launch (results are then undefined) and returns normally.
