@@ -50,11 +50,13 @@ constexpr int kFinisherThreads = kFinisherWarps * 32;
 constexpr int kOffGsum = 2 * kTableBytes;
 constexpr int kOffBar = kOffGsum + 128;
 constexpr int kOffShared = kOffBar + 32;
+constexpr int kOffRecBar = kOffGsum + 192;                // one "record written" barrier per job record
 constexpr int kSlotBytes = 144;                           // descriptor (128) + this CTA's share of the call (16)
 constexpr int kOffDesc = kOffGsum + 256;                  // builders' descriptor ring
 constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // finisher warps: a descriptor ring per warp
 constexpr int kOffJobRec = kOffWarpDesc + kFinisherWarps * kDescSlots * kSlotBytes;   // job records, written by the builders
 constexpr int kJobRecs = 4;
+static_assert(kOffShared + 16 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffDesc, "shared-memory layout");
 constexpr int kChainSmem = kOffJobRec + kJobRecs * 64;
 constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
 constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
@@ -179,6 +181,11 @@ __device__ __forceinline__ void slot_fetch(ChainSlot* dst, const ChainCall* call
 }
 __device__ __forceinline__ uint64_t* bar_full(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + b; }
 __device__ __forceinline__ uint64_t* bar_free(int b) { return reinterpret_cast<uint64_t*>(chain_smem + kOffBar) + 2 + b; }
+// "record of job j is written": one barrier per record slot (the builders are never more than two jobs ahead of the
+// slowest look-up warp, so a slot's barrier cannot run a whole phase ahead of a waiter)
+__device__ __forceinline__ uint64_t* bar_rec(unsigned job) {
+    return reinterpret_cast<uint64_t*>(chain_smem + kOffRecBar) + (job & (kJobRecs - 1));
+}
 
 __device__ __forceinline__ void raise_abort(unsigned* status) {
     ChainShared* sh = chain_shared();
@@ -228,28 +235,28 @@ __device__ __forceinline__ ChainPart chain_part(const ChainSlot* s) {
     return p;
 }
 
-// K-split reduction of call d by this CTA's builder threads: the `groups` CTAs of a row range split its rows;
-// every thread polls the tagged partial sums of its row (all chunks), adds them in ascending chunk order and
-// writes Y.
+// K-split reduction of call d by this CTA's finisher threads.  The `groups` CTAs of a row range share its row blocks
+// round robin (block rb0 + grp, rb0 + grp + groups, ...): the look-up warps produce the blocks of a range in
+// ascending order, so every CTA's share becomes ready evenly over the call and its finishers keep pace with the
+// look-ups instead of starting when the range is nearly done.  A thread owns one row of a block: it polls the row's
+// tagged partial sums (up to 8 chunks in flight), adds them in ascending chunk order and writes Y.
 __device__ __noinline__ void chain_reduce(const ChainCall* d, const ChainPart p, unsigned tag, unsigned limit,
                                           unsigned* status, int ft) {
+    constexpr int kInFlight = 8;
     ChainShared* sh = chain_shared();
-    const int rows = min(p.rb1 * kTileRows, d->N) - p.rb0 * kTileRows;
-    const int per = (rows + d->groups - 1) / d->groups;
-    const int r0 = p.rb0 * kTileRows + p.grp * per;
-    const int r1 = min(p.rb0 * kTileRows + rows, r0 + per);
     const size_t n_pad = (size_t)d->n_rb * kTileRows;
-    const int n_kc = d->n_kc;
-    for (int row = r0 + ft; row < r1; row += kFinisherThreads) {
+    const int n_kc = d->n_kc, N = d->N, stride = d->groups * (kFinisherThreads / kTileRows);
+    for (int rb = p.rb0 + p.grp + d->groups * (ft / kTileRows); rb < p.rb1; rb += stride) {
+        const int row = rb * kTileRows + (ft % kTileRows);
         const unsigned long long* src = d->slots + row;
         float sum = 0.f;
-        for (int c0 = 0; c0 < n_kc; c0 += 8) {
-            unsigned long long v[8];
+        for (int c0 = 0; c0 < n_kc; c0 += kInFlight) {
+            unsigned long long v[kInFlight];
             bool ok = false;
             for (unsigned spin = 0; !ok; ++spin) {
                 ok = true;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < kInFlight; ++i) {
                     if (c0 + i < n_kc) {
                         v[i] = ld_relaxed_u64(src + (size_t)(c0 + i) * n_pad);
                         ok = ok && (unsigned)(v[i] >> 32) == tag;
@@ -262,10 +269,10 @@ __device__ __noinline__ void chain_reduce(const ChainCall* d, const ChainPart p,
                 if (!ok && spin > 64) __nanosleep(64);
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < kInFlight; ++i)
                 if (c0 + i < n_kc) sum += __uint_as_float((unsigned)v[i]);
         }
-        chain_store(d->Y, d->flags, (size_t)row, sum);
+        if (row < N) chain_store(d->Y, d->flags, (size_t)row, sum);
     }
 }
 
@@ -326,13 +333,15 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
     }
 }
 
-// Items of one job on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of the job on entry
-// and, on exit, the item at after_vp (its first item of the next job; nullptr: none).
+// Items of one job on one look-up warp; tables in buffer B.  `buf` holds the warp's first item of the job on entry.
+// At its last item of the job the warp looks for the record of the next job (the builders publish it before they
+// build that job's tables, normally a whole job ahead): if it is there and gives the warp an item, that item's loads
+// ride along with the last item and `buf` holds it on exit (returns true).
 template <int Q, int G, int B>
-__device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
+__device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
                                             unsigned long long* out, void* Y, const int N, const unsigned flags,
-                                            const unsigned tag, const uint8_t* vp, const uint8_t* after_vp, const int lw,
-                                            const int lane) {
+                                            const unsigned tag, const uint8_t* vp, const unsigned job, const size_t warp_off,
+                                            const int lw, const int lane) {
     using C = Cfg<Q, G>;
     const uint8_t* const tab = chain_smem + B * kTableBytes;
     const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
@@ -340,13 +349,20 @@ __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&co
     float S[C::GL];
     load_group_sums<G>(S, gsum, h, l, true);
     const unsigned long long tag_hi = (unsigned long long)tag << 32;
+    bool carried = false;
     for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
-        // next item of this warp: the same job, else the one the caller names
         const bool in_job = rb + kLookupWarps < rb1;
-        const uint8_t* nvp = in_job ? vp + kLookupWarps * C::TILE_BYTES : after_vp;
+        const uint8_t* nvp = vp + kLookupWarps * C::TILE_BYTES;
+        if (!in_job && chain_shared()->recs_published > job + 1) {
+            const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
+            if ((int)n0.z + lw < (int)n0.w) {
+                nvp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + warp_off;
+                carried = true;
+            }
+        }
         const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
         float y;
-        if (in_job || after_vp != nullptr) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
+        if (in_job || carried) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
         else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
         if (h == 0) {
             if (out == nullptr) {
@@ -357,6 +373,7 @@ __device__ __forceinline__ void chain_items(Item<Q, G>& buf, const uint32_t (&co
         }
         vp = nvp;
     }
+    return carried;
 }
 
 // What the roles of a launch share.
@@ -405,11 +422,14 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
     const size_t warp_off = (size_t)lw * C::TILE_BYTES + lane * 16;
     for (unsigned job = 0;; ++job) {
         const int b = job & 1;
-        mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
-        // the job's record in four loads (one round of shared-memory latency instead of a dependent chain of them)
+        // The job's record comes before its tables: the warp requests its first item of the job (unless the item came
+        // along with the job before) and only then waits for the tables, so the two latencies overlap.
+        mbar_wait(bar_rec(job), (job >> 2) & 1, x.spin_limit, x.status);
+        if (sh->abort) break;
+        // the record in four loads (one round of shared-memory latency instead of a dependent chain of them)
         const uint4* rq = reinterpret_cast<const uint4*>(job_rec(job));
         const uint4 q0 = rq[0], q1 = rq[1], q2 = rq[2], q3 = rq[3];
-        if (q3.z != 0u || sh->abort) break;                       // stop record
+        if (q3.z != 0u) break;                                    // stop record
         const uint8_t* tile0 = reinterpret_cast<const uint8_t*>(((unsigned long long)q0.y << 32) | q0.x);
         const int rb0 = (int)q0.z, rb1 = (int)q0.w;
         unsigned long long* out = reinterpret_cast<unsigned long long*>(((unsigned long long)q1.y << 32) | q1.x);
@@ -420,19 +440,10 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
         const bool items = rb0 + lw < rb1;
         const uint8_t* vp = tile0 + warp_off;
         if (items && !carried) load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
-        carried = false;
-        // what follows this warp's last item of the job: its first item of the next job, when that job's record is
-        // already there (the builders normally run a job ahead) and the warp has an item in it
-        const uint8_t* after_vp = nullptr;
-        if (items && sh->recs_published > job + 1) {
-            const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
-            if ((int)n0.z + lw < (int)n0.w) {
-                after_vp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + warp_off;
-                carried = true;
-            }
-        }
-        if (b == 0) chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, after_vp, lw, lane);
-        else chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, after_vp, lw, lane);
+        mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
+        if (sh->abort) break;
+        if (b == 0) carried = chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, job, warp_off, lw, lane);
+        else carried = chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, job, warp_off, lw, lane);
         const bool report = out == nullptr && q3.y != 0u && !(flags & kCallTestNoSignal);
         __syncwarp();
         if (lane == 0) {
@@ -468,18 +479,18 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
 
     // Before any tile is read: the plan is the one the host launched, and every blob of this run still carries
     // the header it was planned with.
+    const int4* parts = reinterpret_cast<const int4*>(reinterpret_cast<const uint8_t*>(ctl) + ctl->parts_off);
+    const int grid = (int)gridDim.x;
+    if (tid < 16 * min(c_end - c_begin, 3)) {     // the first descriptors are on their way while the headers are read
+        const int c = c_begin + (tid >> 4);
+        slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
+    }
     int bad = (ctl->magic != kChainMagic || ctl->n_calls != (unsigned)n_calls) ? 1 : 0;
     if (!bad) {
         for (int c = c_begin + tid; c < c_end; c += kChainThreads) {
             const ChainCall* d = calls + c;
             if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) bad = 1;
         }
-    }
-    const int4* parts = reinterpret_cast<const int4*>(reinterpret_cast<const uint8_t*>(ctl) + ctl->parts_off);
-    const int grid = (int)gridDim.x;
-    if (tid < 16 * min(c_end - c_begin, 3)) {
-        const int c = c_begin + (tid >> 4);
-        slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
     }
     if (tid == 0) {
         sh->abort = 0;
@@ -491,6 +502,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
         mbar_init(bar_full(1), kBuilderWarps);
         mbar_init(bar_free(0), kLookupWarps);
         mbar_init(bar_free(1), kLookupWarps);
+        for (int j = 0; j < kJobRecs; ++j) mbar_init(bar_rec(j), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     cp_async_wait_all();
@@ -564,6 +576,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
                         r->stop = 0;
                         __threadfence_block();
                         sh->recs_published = job + 1;
+                        mbar_arrive(bar_rec(job));
                     }
                     if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);   // look-ups of job - 2 are over
                     build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), xv, bw, lane);
@@ -591,6 +604,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
                 r->stop = 1;
                 __threadfence_block();
                 sh->recs_published = job + 1;
+                mbar_arrive(bar_rec(job));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_full(b));
