@@ -56,8 +56,14 @@ constexpr int kOffDesc = kOffGsum + 256;                  // builders' descripto
 constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // finisher warps: a descriptor ring per warp
 constexpr int kOffJobRec = kOffWarpDesc + kFinisherWarps * kDescSlots * kSlotBytes;   // job records, written by the builders
 constexpr int kJobRecs = 4;
-static_assert(kOffShared + 16 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffDesc, "shared-memory layout");
-constexpr int kChainSmem = kOffJobRec + kJobRecs * 64;
+static_assert(kOffShared + 32 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffDesc, "shared-memory layout");
+// finisher warps: a ring of buffers per warp that bulk copies fill with the partial sums of one row block
+constexpr int kFinSlots = 2;                  // copies in flight per finisher warp (measured on the 8B step and the
+                                              // 32-layer stack: 1: 77.8 / 562 us, 2: 79.1 / 541 us, 4: 82.7 / 580 us, 8: 88 / 651 us)
+constexpr int kFinRingBytes = 8192;           // per warp: one buffer of 32 chunks per slot
+constexpr int kOffFinBuf = (kOffJobRec + kJobRecs * 64 + 127) / 128 * 128;
+constexpr int kOffFinBar = kOffFinBuf + kFinisherWarps * kFinRingBytes;
+constexpr int kChainSmem = kOffFinBar + kFinisherWarps * kFinSlots * 8;
 constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
 constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
 
@@ -71,7 +77,7 @@ struct ChainCall {                            // 128 bytes
     const __half* X;
     const uint8_t* tiles;                     // packed + header
     void* Y;
-    unsigned long long* slots;                // [n_kc][n_rb * 16] tagged partial sums of this call's scratch region
+    unsigned long long* slots;                // [n_rb][n_kc][16] tagged partial sums of this call's scratch region
     int N, K, n_rb, n_kc;
     int q, G;
     unsigned flags;
@@ -92,11 +98,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
@@ -112,6 +113,9 @@ __device__ __forceinline__ void cp_async_wait_all() {
 }
 __device__ __forceinline__ void bar_builders() {          // named barrier 1: the builder warps only
     asm volatile("bar.sync 1, %0;" ::"n"(kBuilderThreads) : "memory");
+}
+__device__ __forceinline__ void bar_lookups() {           // named barrier 3: the look-up warps only
+    asm volatile("bar.sync 3, %0;" ::"n"(kLookupWarps * 32) : "memory");
 }
 __device__ __forceinline__ void bar_finishers() {         // named barrier 2: the finisher warps only
     asm volatile("bar.sync 2, %0;" ::"n"(kFinisherThreads) : "memory");
@@ -135,14 +139,16 @@ struct ChainShared {
     volatile int abort;                       // a wait ran out: stop waiting
     unsigned epoch;
     volatile unsigned recs_published;         // job records written so far (by the builders)
+    volatile int headers_bad;                 // a blob of this launch no longer carries the header it was planned with
 };
+static_assert(sizeof(ChainShared) <= 32, "shared flags");
 
 // What the look-up warps need to know of one table job (a call's K chunk on this CTA), written by the builders
 // before they build the job's tables: the look-up warps follow these records and never touch a descriptor.
 struct JobRec {                               // four 16-byte quarters, each read with one shared-memory load
     const uint8_t* tile0;                     // the job's first item (row block rb0 of chunk kc)
     int rb0, rb1;                             //   (a record with rb0 == rb1 has no items: the stop record)
-    unsigned long long* out;                  // tagged partial sums of chunk kc (row 0), or nullptr: no K split, store Y
+    unsigned long long* out;                  // tagged partial sums of chunk kc (row block 0), or nullptr: no K split, store Y
     void* Y;
     unsigned* done;                           // completion counter of the call (used without a K split)
     int N;
@@ -150,7 +156,7 @@ struct JobRec {                               // four 16-byte quarters, each rea
     unsigned tag;
     int last;                                 // 1: the call's last job on this CTA
     int stop;                                 // 1: no more jobs in this launch
-    int pad;
+    int out_stride;                           // 64-bit words from one row block's partial sums to the next (16 n_kc)
 };
 static_assert(sizeof(JobRec) == 64, "job record size");
 
@@ -235,45 +241,138 @@ __device__ __forceinline__ ChainPart chain_part(const ChainSlot* s) {
     return p;
 }
 
-// K-split reduction of call d by this CTA's finisher threads.  The `groups` CTAs of a row range share its row blocks
-// round robin (block rb0 + grp, rb0 + grp + groups, ...): the look-up warps produce the blocks of a range in
-// ascending order, so every CTA's share becomes ready evenly over the call and its finishers keep pace with the
-// look-ups instead of starting when the range is nearly done.  A thread owns one row of a block: it polls the row's
-// tagged partial sums (up to 8 chunks in flight), adds them in ascending chunk order and writes Y.
-__device__ __noinline__ void chain_reduce(const ChainCall* d, const ChainPart p, unsigned tag, unsigned limit,
-                                          unsigned* status, int ft) {
-    constexpr int kInFlight = 8;
+// Bulk copy global -> shared memory, completion counted in bytes on a shared-memory barrier (both addresses and
+// the size are multiples of 16 bytes).
+__device__ __forceinline__ void fin_copy(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src), "r"(bytes), "r"(b) : "memory");
+}
+__device__ __forceinline__ uint64_t* fin_bar(int fw, int slot) {
+    return reinterpret_cast<uint64_t*>(chain_smem + kOffFinBar) + fw * kFinSlots + slot;
+}
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+    // one fire-and-forget instruction: the writes that happen before it (this thread's, and those of the threads it
+    // has synchronised with at a barrier) are visible to whoever reads the new count with acquire semantics
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity) {     // one look, no suspension
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// K-split reduction of call d by one finisher warp.  The `groups` CTAs of a row range share its row blocks round
+// robin (block rb0 + grp, rb0 + grp + groups, ...): the look-up warps produce the blocks of a range in ascending
+// order, so every CTA's share becomes ready evenly over the call and its finishers keep pace with the look-ups.
+// The CTA's blocks alternate between its finisher warps.  The partial sums of a row block lie together
+// ([chunk][16 rows], 128 bytes per chunk), so one bulk copy brings a block's sums (in segments of 32 chunks, when
+// there are more) into shared memory without holding a register.  The warp's D = kFinSlots ring slots work on D
+// blocks independently (slot k on the warp's blocks k, k + D, ...): when a slot's copy has landed, lane l < 16 adds
+// row l's sums in ascending chunk order and checks their tags; if one is not this call's yet, the same copy is issued
+// again, otherwise the slot's next copy.  A load issued on an SM whose look-up warps keep ~60 KB of weight loads
+// outstanding comes back only after thousands of cycles (measured: ~5000), so what the finishers need is polls in
+// flight, not instructions: with per-thread polling loads (8 in flight per thread) the reduction of a call took as
+// long as its look-ups on every shape with more than a few row blocks per CTA.  `phases` holds the barrier parities
+// of the warp's slots across calls.  Bounded: `limit` sweeps over the ring without a complete copy end the launch
+// with the wait-expired status.
+__device__ __noinline__ unsigned chain_reduce(const ChainCall* d, const ChainPart p, unsigned tag, unsigned limit,
+                                              unsigned* status, int fw, int lane, unsigned phases) {
     ChainShared* sh = chain_shared();
-    const size_t n_pad = (size_t)d->n_rb * kTileRows;
-    const int n_kc = d->n_kc, N = d->N, stride = d->groups * (kFinisherThreads / kTileRows);
-    for (int rb = p.rb0 + p.grp + d->groups * (ft / kTileRows); rb < p.rb1; rb += stride) {
-        const int row = rb * kTileRows + (ft % kTileRows);
-        const unsigned long long* src = d->slots + row;
-        float sum = 0.f;
-        for (int c0 = 0; c0 < n_kc; c0 += kInFlight) {
-            unsigned long long v[kInFlight];
-            bool ok = false;
-            for (unsigned spin = 0; !ok; ++spin) {
-                ok = true;
+    const int n_kc = d->n_kc, N = d->N, groups = d->groups;
+    constexpr int D = kFinSlots;                               // ring slots in use
+    constexpr int seg_chunks = 32, buf_bytes = kFinRingBytes / D;
+    const int nseg = (n_kc + seg_chunks - 1) / seg_chunks;
+    const int first = p.rb0 + p.grp + fw * groups;             // this warp's first block
+    const int nblk = first < p.rb1 ? (p.rb1 - first + kFinisherWarps * groups - 1) / (kFinisherWarps * groups) : 0;
+    uint8_t* const ring = chain_smem + kOffFinBuf + fw * kFinRingBytes;
+    unsigned pending = 0;                                      // ring slots with a copy in flight
+    auto issue = [&](int slot, int j, int sg) {                // segment sg of the warp's block j
+        const int rb = first + j * kFinisherWarps * groups;
+        const int nch = min(seg_chunks, n_kc - sg * seg_chunks);
+        if (lane == 0)
+            fin_copy(ring + slot * buf_bytes, d->slots + ((size_t)rb * n_kc + (size_t)sg * seg_chunks) * kTileRows,
+                     (unsigned)nch * kTileRows * 8, fin_bar(fw, slot));
+        pending |= 1u << slot;
+    };
+    int blk[kFinSlots], seg[kFinSlots];
+    float sums[kFinSlots];
 #pragma unroll
-                for (int i = 0; i < kInFlight; ++i) {
-                    if (c0 + i < n_kc) {
-                        v[i] = ld_relaxed_u64(src + (size_t)(c0 + i) * n_pad);
-                        ok = ok && (unsigned)(v[i] >> 32) == tag;
-                    }
-                }
-                if (!ok && (spin >= limit || sh->abort)) {
-                    raise_abort(status);
-                    break;
-                }
-                if (!ok && spin > 64) __nanosleep(64);
-            }
-#pragma unroll
-            for (int i = 0; i < kInFlight; ++i)
-                if (c0 + i < n_kc) sum += __uint_as_float((unsigned)v[i]);
-        }
-        if (row < N) chain_store(d->Y, d->flags, (size_t)row, sum);
+    for (int k = 0; k < kFinSlots; ++k) {
+        blk[k] = k < D ? k : nblk;                             // (slots beyond D stay idle)
+        seg[k] = 0; sums[k] = 0.f;
     }
+#pragma unroll
+    for (int k = 0; k < kFinSlots; ++k)
+        if (blk[k] < nblk) issue(k, blk[k], 0);
+    int remaining = nblk;
+    unsigned idle = 0;
+    while (remaining > 0) {
+        bool progress = false, accepted = false;               // a copy has landed; a landed copy was complete
+#pragma unroll
+        for (int k = 0; k < kFinSlots; ++k) {
+            if (blk[k] >= nblk) continue;
+            if (!__all_sync(0xffffffffu, mbar_test(fin_bar(fw, k), (phases >> k) & 1u))) continue;
+            phases ^= 1u << k;
+            pending &= ~(1u << k);
+            progress = true;
+            const int rb = first + blk[k] * kFinisherWarps * groups;
+            const int nch = min(seg_chunks, n_kc - seg[k] * seg_chunks);
+            const unsigned long long* buf = reinterpret_cast<const unsigned long long*>(ring + k * buf_bytes);
+            bool ok = true;
+            float part = 0.f;
+            if (lane < kTileRows) {
+                for (int c = 0; c < nch; ++c) {
+                    const unsigned long long w = buf[c * kTileRows + lane];
+                    ok = ok && (unsigned)(w >> 32) == tag;
+                    part += __uint_as_float((unsigned)w);
+                }
+            }
+            if (__all_sync(0xffffffffu, ok)) {                  // (also: every lane is done with the buffer)
+                sums[k] = seg[k] == 0 ? part : sums[k] + part;
+                if (seg[k] + 1 == nseg) {
+                    const int row = rb * kTileRows + lane;
+                    if (lane < kTileRows && row < N) chain_store(d->Y, d->flags, (size_t)row, sums[k]);
+                    blk[k] += D;
+                    seg[k] = 0;
+                    remaining -= 1;
+                } else {
+                    seg[k] += 1;
+                }
+                accepted = true;
+            }
+            // the slot's next copy, or the same one again when some of its sums were not there yet
+            if (blk[k] < nblk) issue(k, blk[k], seg[k]);
+        }
+        if (accepted) {
+            idle = 0;
+        } else {
+            if (++idle > limit || sh->abort) {
+                raise_abort(status);
+                break;
+            }
+            if (!progress) {
+                // nothing has landed: wait for one of the copies suspended by the hardware (about a microsecond at
+                // most per attempt) instead of sweeping, which would take issue slots from the look-up warps
+                const int k0 = __ffs(pending) - 1;
+                mbar_try(fin_bar(fw, k0), (phases >> k0) & 1u);
+            }
+        }
+    }
+    // a warp that gives up still waits (bounded, without looking at the abort flag) for its copies in flight: the
+    // shared memory they write to must not be handed to another CTA before they have landed
+#pragma unroll
+    for (int k = 0; k < kFinSlots; ++k) {
+        if (pending & (1u << k)) {
+            bool landed = false;
+            for (int tries = 0; tries < 4096 && !landed; ++tries) landed = mbar_try(fin_bar(fw, k), (phases >> k) & 1u);
+            phases ^= 1u << k;
+        }
+    }
+    return phases;
 }
 
 // The lane's 16 activations of chunk kc (two byte-columns), as (x_i of column 2*lane, x_i of column 2*lane+1).
@@ -340,8 +439,8 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 template <int Q, int G, int B>
 __device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
                                             unsigned long long* out, void* Y, const int N, const unsigned flags,
-                                            const unsigned tag, const uint8_t* vp, const unsigned job, const size_t warp_off,
-                                            const int lw, const int lane) {
+                                            const unsigned tag, const int out_stride, const uint8_t* vp, const unsigned job,
+                                            const size_t warp_off, const int lw, const int lane) {
     using C = Cfg<Q, G>;
     const uint8_t* const tab = chain_smem + B * kTableBytes;
     const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
@@ -368,7 +467,7 @@ __device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&co
             if (out == nullptr) {
                 if (rb * kTileRows + l < N) chain_store(Y, flags, (size_t)(rb * kTileRows + l), y);
             } else {
-                st_relaxed_u64(out + rb * kTileRows + l, tag_hi | __float_as_uint(y));
+                st_relaxed_u64(out + (size_t)rb * out_stride + l, tag_hi | __float_as_uint(y));
             }
         }
         vp = nvp;
@@ -437,22 +536,19 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
         unsigned* done_c = reinterpret_cast<unsigned*>(((unsigned long long)q2.y << 32) | q2.x);
         const int N = (int)q2.z;
         const unsigned flags = q2.w, tag = q3.x;
+        const int out_stride = (int)q3.w;
         const bool items = rb0 + lw < rb1;
         const uint8_t* vp = tile0 + warp_off;
         if (items && !carried) load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
         mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
         if (sh->abort) break;
-        if (b == 0) carried = chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, job, warp_off, lw, lane);
-        else carried = chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, vp, job, warp_off, lw, lane);
+        if (b == 0) carried = chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
+        else carried = chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
         const bool report = out == nullptr && q3.y != 0u && !(flags & kCallTestNoSignal);
         __syncwarp();
         if (lane == 0) {
             mbar_arrive(bar_free(b));         // this warp no longer reads buffer b (nor the job's record)
-            if (report) {
-                // no K split: this warp stored its rows of Y itself and reports them
-                __threadfence();
-                atomicAdd(done_c, 1u);
-            }
+            if (report) red_release_add(done_c, 1u);     // no K split: this warp stored its rows of Y itself and reports them
         }
     }
 }
@@ -460,11 +556,10 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
 // Calls [c_begin, c_end) of the plan, all with the kernel's (Q, G).
 template <int Q, int G>
 __global__ void __launch_bounds__(kChainThreads, 1)
-lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const int c_begin, const int c_end,
-                 const int first_run, const int last_run, const unsigned spin_limit) {
+lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsigned* done, const int n_calls,
+                 const int c_begin, const int c_end, const int first_run, const int last_run, const unsigned spin_limit) {
     uint8_t* const smem = chain_smem;
     ChainShared* sh = chain_shared();
-    unsigned* done = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(ctl) + ctl->done_off);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bid = blockIdx.x;
 
@@ -477,25 +572,22 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
     if (first_run) grid_dependency_wait();
     grid_launch_dependents();
 
-    // Before any tile is read: the plan is the one the host launched, and every blob of this run still carries
-    // the header it was planned with.
-    const int4* parts = reinterpret_cast<const int4*>(reinterpret_cast<const uint8_t*>(ctl) + ctl->parts_off);
+    // The plan is the one the host launched (its parts are addressed through kernel arguments: no pointer is
+    // chased through the control block on the way to the first descriptor).
     const int grid = (int)gridDim.x;
-    if (tid < 16 * min(c_end - c_begin, 3)) {     // the first descriptors are on their way while the headers are read
+    if (tid < 16 * min(c_end - c_begin, 3)) {
         const int c = c_begin + (tid >> 4);
         slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
     }
-    int bad = (ctl->magic != kChainMagic || ctl->n_calls != (unsigned)n_calls) ? 1 : 0;
-    if (!bad) {
-        for (int c = c_begin + tid; c < c_end; c += kChainThreads) {
-            const ChainCall* d = calls + c;
-            if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) bad = 1;
-        }
-    }
+    unsigned epoch_now = 0;
+    int bad = 0;
     if (tid == 0) {
+        bad = (ctl->magic != kChainMagic || ctl->n_calls != (unsigned)n_calls) ? 1 : 0;
+        epoch_now = ctl->epoch;
         sh->abort = 0;
+        sh->headers_bad = 0;
         sh->recs_published = 0;
-        sh->epoch = ctl->epoch;
+        sh->epoch = epoch_now;
         // one arrival per warp (its lane 0, after the warp has converged): 32 arrivals of a warp on one barrier word
         // would be 32 serialised shared-memory atomics
         mbar_init(bar_full(0), kBuilderWarps);
@@ -503,6 +595,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
         mbar_init(bar_free(0), kLookupWarps);
         mbar_init(bar_free(1), kLookupWarps);
         for (int j = 0; j < kJobRecs; ++j) mbar_init(bar_rec(j), 1);
+        for (int j = 0; j < kFinisherWarps * kFinSlots; ++j) mbar_init(fin_bar(0, j), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     cp_async_wait_all();
@@ -512,6 +605,14 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
     }
     const unsigned epoch = sh->epoch;
     unsigned* const status = &ctl->status;
+    if (tid == 0 && last_run) {
+        // The CTA of the chain's last launch that starts last opens the next epoch (completion counters and tags keep
+        // counting up across launches of a plan, so nothing has to be cleared).  Every CTA of this launch has read the
+        // epoch before it takes its ticket, and when all of them have started every CTA of the launches before has
+        // left; the next run of the plan reads the epoch only after this launch has completed (stream order).
+        const unsigned t = atomicInc(&ctl->exit_ticket, gridDim.x - 1);
+        if (t == gridDim.x - 1) ctl->epoch = epoch + 1u;
+    }
 
     ChainCtx x;
     x.calls = calls; x.parts = parts; x.done = done; x.status = status;
@@ -520,7 +621,26 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
 
     if (warp < kLookupWarps) {
         // ---------------------------------------------------------------- look-up warps
-        lookup_jobs<Q, G>(x);
+        // Before any tile is read: every blob of this launch still carries the header it was planned with.  Only
+        // the look-up warps read tiles, so only they wait for the headers; the builders fetch activations and build
+        // the first tables meanwhile.
+        {
+            int hdr_bad = 0;
+            for (int c = c_begin + tid; c < c_end; c += kLookupWarps * 32) {
+                const ChainCall* d = calls + c;
+                if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) hdr_bad = 1;
+            }
+            if (hdr_bad) sh->headers_bad = 1;
+            bar_lookups();
+            if (sh->headers_bad) {
+                if (tid == 0) {
+                    sh->abort = 1;            // the other roles' waits end at their next look at this flag
+                    atomicExch(status, kStatusBlobMismatch);
+                }
+            } else {
+                lookup_jobs<Q, G>(x);
+            }
+        }
     } else if (warp < kLookupWarps + kBuilderWarps) {
         // ---------------------------------------------------------------- builder warps
         const int bw = warp - kLookupWarps, bt = tid - kLookupWarps * 32;
@@ -566,7 +686,8 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
                         JobRec* r = job_rec(job);
                         const int kc = p.kc0 + seg;
                         r->tile0 = d->tiles + ((size_t)kc * d->n_rb + p.rb0) * Cfg<Q, G>::TILE_BYTES;
-                        r->out = d->n_kc > 1 ? d->slots + (size_t)kc * ((size_t)d->n_rb * kTileRows) : nullptr;
+                        r->out = d->n_kc > 1 ? d->slots + (size_t)kc * kTileRows : nullptr;
+                        r->out_stride = d->n_kc * kTileRows;
                         r->Y = d->Y;
                         r->done = done + c;
                         r->rb0 = p.rb0; r->rb1 = p.rb1; r->N = d->N;
@@ -613,6 +734,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
         // ---------------------------------------------------------------- finisher warps
         // K-split reduction of every call this CTA works on, then the call's completion report
         const int fw = warp - kLookupWarps - kBuilderWarps, ft = tid - (kLookupWarps + kBuilderWarps) * 32;
+        unsigned phases = 0;                  // parities of this warp's copy barriers
         desc_begin(x, fw, lane);
         for (int c = c_begin; c < c_end; ++c) {
             const ChainSlot* sl = desc_next(x, fw, c, lane);
@@ -620,26 +742,12 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int n_calls, const
             if (bid < d->n_ctas && d->n_kc > 1) {
                 const ChainPart p = chain_part(sl);
                 const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
-                chain_reduce(d, p, tag, spin_limit, status, ft);
+                phases = chain_reduce(d, p, tag, spin_limit, status, fw, lane, phases);
                 bar_finishers();              // every row of this CTA is stored
-                if (ft == 0 && !(d->flags & kCallTestNoSignal)) {
-                    __threadfence();
-                    atomicAdd(done + c, 1u);
-                }
+                if (ft == 0 && !(d->flags & kCallTestNoSignal)) red_release_add(done + c, 1u);
             }
             __syncwarp();
         }
-        // the CTA that leaves the chain's last launch last opens the next epoch (completion counters and tags keep
-        // counting up across launches, so nothing has to be cleared); the finishers are the last of a CTA to be done
-        // with a call whose sums are split over K, the look-up warps with one that is not: both are waited for
-        bar_finishers();
-    }
-    __syncthreads();
-    if (tid == 0 && last_run) {
-        // (when every CTA of the chain's last launch has started, every CTA of the launches before it has left)
-        __threadfence();
-        const unsigned t = atomicInc(&ctl->exit_ticket, gridDim.x - 1);
-        if (t == gridDim.x - 1) ctl->epoch = epoch + 1u;
     }
 }
 
@@ -679,8 +787,8 @@ int check_call(const elutq_gemv_call& c) {
 }
 
 template <int Q, int G>
-cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int first_run, int last_run,
-                       unsigned wait_limit, int sms, cudaStream_t stream) {
+cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsigned* done, int n_calls, int c0, int c1,
+                       int first_run, int last_run, unsigned wait_limit, int sms, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -707,18 +815,18 @@ cudaError_t launch_run(ChainCtl* ctl, const ChainCall* calls, int n_calls, int c
     // as SMs - so all of them become resident as soon as the predecessor has drained, and every wait is bounded.
     cfg.attrs = first_run ? attr : attr + 1;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, lut_chain_kernel<Q, G>, ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit);
+    e = cudaLaunchKernelEx(&cfg, lut_chain_kernel<Q, G>, ctl, calls, parts, done, n_calls, c0, c1, first_run, last_run, wait_limit);
     count_launch(1);
     return e;
 }
 
 template <int Q>
-cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, int n_calls, int c0, int c1, int first_run, int last_run,
-                         unsigned wait_limit, int sms, cudaStream_t stream) {
+cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsigned* done, int n_calls, int c0,
+                         int c1, int first_run, int last_run, unsigned wait_limit, int sms, cudaStream_t stream) {
     switch (G) {
-        case 128: return launch_run<Q, 128>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
-        case 64: return launch_run<Q, 64>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
-        case 32: return launch_run<Q, 32>(ctl, calls, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
+        case 128: return launch_run<Q, 128>(ctl, calls, parts, done, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
+        case 64: return launch_run<Q, 64>(ctl, calls, parts, done, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
+        case 32: return launch_run<Q, 32>(ctl, calls, parts, done, n_calls, c0, c1, first_run, last_run, wait_limit, sms, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -730,7 +838,7 @@ struct PlanRuns {
     int n_runs = 0;
     int begin[kMaxRuns + 1] = {};
     int q[kMaxRuns] = {}, G[kMaxRuns] = {};
-    size_t calls_off = 0;
+    size_t calls_off = 0, parts_off = 0, done_off = 0;
 };
 std::mutex g_plan_mu;
 std::map<const void*, PlanRuns> g_plans;
@@ -773,7 +881,7 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
     ChainCall* dc = reinterpret_cast<ChainCall*>(host.data() + L.calls_off);
     PlanRuns runs;
     runs.n_calls = n_calls;
-    runs.calls_off = L.calls_off;
+    runs.calls_off = L.calls_off; runs.parts_off = L.parts_off; runs.done_off = L.done_off;
     for (int i = 0; i < n_calls; ++i) {
         const elutq_gemv_call& c = calls[i];
         int q = 0, G = 0;
@@ -859,16 +967,18 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* str
     }
     ChainCtl* ctl = reinterpret_cast<ChainCtl*>(plan);
     const ChainCall* calls = reinterpret_cast<const ChainCall*>(reinterpret_cast<uint8_t*>(plan) + runs.calls_off);
+    const int4* parts = reinterpret_cast<const int4*>(reinterpret_cast<uint8_t*>(plan) + runs.parts_off);
+    unsigned* done = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(plan) + runs.done_off);
     if (wait_limit == 0) wait_limit = 1u << 22;
     const int sms = device_sm_count();
     for (int r = 0; r < runs.n_runs; ++r) {
         const int last = r + 1 == runs.n_runs;
         cudaError_t e;
         switch (runs.q[r]) {
-            case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
-            case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
-            case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
-            case 4: e = launch_run_q<4>(runs.G[r], ctl, calls, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
+            case 4: e = launch_run_q<4>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
             default: e = cudaErrorInvalidValue; break;
         }
         if (e != cudaSuccess) return note_cuda_error((int)e);

@@ -24,10 +24,11 @@ from gpu_util import pack_layer, x_dev  # noqa: E402
 TOL_F32 = 5e-6
 TOL_F16 = 1e-3
 
-# (q, G, N, K): every q, every G, ragged rows, one-chunk layers (no K split), many chunks, several chunks per CTA
+# (q, G, N, K): every q, every G, ragged rows, one-chunk layers (no K split), many chunks, several chunks per CTA,
+# chunk counts that give one, two and four finisher threads per output row (up to 8, 9-16, more chunks)
 SHAPES = [(2, 128, 100, 1024), (3, 128, 333, 1536), (4, 128, 64, 2560), (2, 64, 50, 1088), (1, 32, 17, 96),
           (2, 128, 16, 512), (3, 64, 1000, 4096), (4, 32, 48, 1024), (1, 128, 1, 128), (2, 128, 5000, 4096),
-          (2, 128, 40, 512 * 160)]
+          (2, 128, 40, 512 * 160), (3, 128, 100, 6144), (4, 64, 300, 512 * 20)]
 
 
 def _elementwise_ok(y, ref, rel):
