@@ -169,11 +169,19 @@ constexpr unsigned kFlagTestNoMma = 0x20000000u;   // the blob header does not d
 // past the end of the buffer.  `tiles` points just behind the 128-byte header.  On mismatch the status word is
 // raised and the caller returns without touching the tiles (every thread sees the same header, so a CTA
 // leaves as a whole).
+__device__ __forceinline__ void blob_header_load(const uint8_t* tiles, uint4& h0, uint2& h1) {
+    h0 = __ldg(reinterpret_cast<const uint4*>(tiles - ELUTQ_HEADER_BYTES));
+    h1 = __ldg(reinterpret_cast<const uint2*>(tiles - ELUTQ_HEADER_BYTES + 16));
+}
+__device__ __forceinline__ bool blob_header_ok(const uint4& h0, const uint2& h1, int q, int G, int N, int K) {
+    return h0.x == (uint32_t)kMagic && h0.y == (uint32_t)kVersion && h0.z == (uint32_t)q && h0.w == (uint32_t)G &&
+           h1.x == (uint32_t)N && h1.y == (uint32_t)K;
+}
 __device__ __forceinline__ bool blob_header_matches(const uint8_t* tiles, int q, int G, int N, int K, unsigned* status) {
-    const uint4 h0 = __ldg(reinterpret_cast<const uint4*>(tiles - ELUTQ_HEADER_BYTES));
-    const uint2 h1 = __ldg(reinterpret_cast<const uint2*>(tiles - ELUTQ_HEADER_BYTES + 16));
-    const bool ok = h0.x == (uint32_t)kMagic && h0.y == (uint32_t)kVersion && h0.z == (uint32_t)q && h0.w == (uint32_t)G &&
-                    h1.x == (uint32_t)N && h1.y == (uint32_t)K;
+    uint4 h0;
+    uint2 h1;
+    blob_header_load(tiles, h0, h1);
+    const bool ok = blob_header_ok(h0, h1, q, G, N, K);
     if (!ok && status != nullptr && threadIdx.x == 0) atomicExch(status, kStatusBlobMismatch);
     return ok;
 }

@@ -579,6 +579,19 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         const int c = c_begin + (tid >> 4);
         slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
     }
+    // Header check, first part: the look-up threads 64, 65, ... read the header of one call's blob each.  The loads
+    // are issued here and looked at after the barrier below, so that they are on their way while the descriptors
+    // arrive (the check needs a call's descriptor first: two loads behind one another).
+    constexpr int kHdrFirst = 64, kHdrThreads = kLookupWarps * 32 - kHdrFirst;
+    uint4 hdr0 = make_uint4(0, 0, 0, 0);
+    uint2 hdr1 = make_uint2(0, 0);
+    int hdr_q = 0, hdr_g = 0, hdr_n = 0, hdr_k = 0;
+    const bool hdr_mine = tid >= kHdrFirst && tid < kLookupWarps * 32 && c_begin + (tid - kHdrFirst) < c_end;
+    if (hdr_mine) {
+        const ChainCall* d = calls + c_begin + (tid - kHdrFirst);
+        hdr_q = d->q; hdr_g = d->G; hdr_n = d->N; hdr_k = d->K;
+        blob_header_load(d->tiles, hdr0, hdr1);
+    }
     unsigned epoch_now = 0;
     int bad = 0;
     if (tid == 0) {
@@ -626,7 +639,8 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         // the first tables meanwhile.
         {
             int hdr_bad = 0;
-            for (int c = c_begin + tid; c < c_end; c += kLookupWarps * 32) {
+            if (hdr_mine && (hdr_q != Q || hdr_g != G || !blob_header_ok(hdr0, hdr1, Q, G, hdr_n, hdr_k))) hdr_bad = 1;
+            for (int c = c_begin + kHdrThreads + tid; c < c_end; c += kLookupWarps * 32) {      // launches of more calls
                 const ChainCall* d = calls + c;
                 if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) hdr_bad = 1;
             }
