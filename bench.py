@@ -645,6 +645,39 @@ def run_cuda(args) -> None:
                                  "frac_of_hbm_peak": round(b / max(us, 1e-3) / 1e3 / peak, 3),
                                  "tflop_eq": round(2.0 * c.M * c.N * c.K / max(us, 1e-3) / 1e6, 3),
                                  "how": "marginal time of one extra separate call inside the graph-replayed step"})
+                if c.M == 1:
+                    # the same shape inside the chained entry: a chain of n copies of the layer (own blobs, so every
+                    # call streams from HBM) against a chain of one, per extra call
+                    n_in = 9
+                    clones = [clone] + [l["packed"].clone() for _ in range(n_in - 1)]
+                    for cl in clones[1:]:
+                        elutq.elutq_describe(cl, c.N, c.K)
+                    Ys = [torch.empty_like(l["Y"]) for _ in range(n_in)]
+                    plan_n = elutq.elutq_chain_plan([(l["X"], clones[i], Ys[i], c.N, c.K) for i in range(n_in)])
+                    plan_1 = elutq.elutq_chain_plan([(l["X"], clones[0], Ys[0], c.N, c.K)])
+
+                    def time_chain(plan, n):
+                        for _ in range(3):
+                            elutq.elutq_chain_run(plan, n, stream=stream)
+                        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a0.record(stream)
+                        for _ in range(reps_pc):
+                            elutq.elutq_chain_run(plan, n, stream=stream)
+                        a1.record(stream)
+                        stream.synchronize()
+                        return a0.elapsed_time(a1) * 1e3 / reps_pc
+
+                    us_c = max(time_chain(plan_n, n_in) - time_chain(plan_1, 1), 0.0) / (n_in - 1)
+                    per_call[-1].update({"us_in_chain": round(us_c, 3),
+                                         "frac_of_hbm_peak_in_chain": round(b / max(us_c, 1e-3) / 1e3 / peak, 3),
+                                         "how_in_chain": "(chain of 9 copies of the layer - chain of 1) / 8, elutq_chain_run"})
+                    if elutq.elutq_chain_status(plan_n) or elutq.elutq_chain_status(plan_1):
+                        per_call[-1]["in_chain_device_status"] = [elutq.elutq_chain_status(plan_n), elutq.elutq_chain_status(plan_1)]
+                    elutq.elutq_chain_forget(plan_n)
+                    elutq.elutq_chain_forget(plan_1)
+                    for cl in clones[1:]:
+                        elutq.elutq_forget(cl)
+                    del clones, Ys, plan_n, plan_1
                 elutq.elutq_forget(clone)
                 del g2, clone, Y2
 
