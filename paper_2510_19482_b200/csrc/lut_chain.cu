@@ -15,17 +15,19 @@
 //     entries.  Buffers are handed over through shared-memory mbarriers ("full" / "free" per buffer, one arrival per
 //     warp, waits suspended in hardware rather than spinning);
 //   * K split: every partial sum is stored together with a tag (launch epoch and call number) in one 8-byte
-//     word.  The CTAs that share a row range split its rows among themselves; 2 finisher warps poll (bounded) the
-//     tagged words of their rows, add the chunks in ascending order - bit-reproducible - and write Y, then report
-//     the call's completion on a counter.  No fence, no ticket, no second kernel for the reduction: the load that
-//     finds the tag is the load that brings the value.
+//     word, all sums of a row block side by side ([row block][chunk][16 rows]).  The CTAs that share a row range take
+//     its row blocks round robin; each of the CTA's 2 finisher warps brings a block's sums into shared memory with
+//     one bulk copy (two copies in flight per warp, completion on an mbarrier), adds the chunks in ascending order -
+//     bit-reproducible -, checks the tags, repeats the copy (bounded) while a tag is not this call's yet, writes Y
+//     and reports the call's completion on a counter.  No fence, no ticket, no second kernel for the reduction: the
+//     copy that finds the tags is the copy that brings the values.
 //   * Ordering: the result is what the calls give when run one after another.  The plan records, from the buffer
 //     addresses, which earlier calls a call really depends on (its X or Y overlaps their Y, or its Y their X);
 //     before the builders read X they wait (bounded) for the completion counters of exactly those calls.  Calls
 //     without such a dependency overlap freely, so the weight stream does not stop at call boundaries.
 //
-// Every wait is a bounded poll; when one runs out the CTA raises the plan's status word, stops waiting for
-// the rest of the launch (results are then undefined) and returns normally.
+// Every wait is bounded; when one runs out the CTA raises the plan's status word, stops waiting for the rest of the
+// launch (results are then undefined), waits (bounded) for its own bulk copies in flight and returns normally.
 #include <cstring>
 #include <map>
 #include <mutex>
