@@ -646,38 +646,43 @@ def run_cuda(args) -> None:
                                  "tflop_eq": round(2.0 * c.M * c.N * c.K / max(us, 1e-3) / 1e6, 3),
                                  "how": "marginal time of one extra separate call inside the graph-replayed step"})
                 if c.M == 1:
-                    # the same shape inside the chained entry: a chain of n copies of the layer (own blobs, so every
-                    # call streams from HBM) against a chain of one, per extra call
+                    # the same shape inside the chained entry: chains of n copies of the layer against chains of one, per
+                    # extra call; the launches rotate over enough distinct blobs (more than twice the L2) that every
+                    # call streams from HBM
                     n_in = 9
-                    clones = [clone] + [l["packed"].clone() for _ in range(n_in - 1)]
-                    for cl in clones[1:]:
+                    n_plans = max(2, -(-(2 * l2_bytes + (64 << 20)) // (n_in * l["packed"].numel())))
+                    clones = [l["packed"].clone() for _ in range(n_plans * n_in)]
+                    for cl in clones:
                         elutq.elutq_describe(cl, c.N, c.K)
                     Ys = [torch.empty_like(l["Y"]) for _ in range(n_in)]
-                    plan_n = elutq.elutq_chain_plan([(l["X"], clones[i], Ys[i], c.N, c.K) for i in range(n_in)])
-                    plan_1 = elutq.elutq_chain_plan([(l["X"], clones[0], Ys[0], c.N, c.K)])
+                    plans_n = [elutq.elutq_chain_plan([(l["X"], clones[s_ * n_in + i], Ys[i], c.N, c.K) for i in range(n_in)])
+                               for s_ in range(n_plans)]
+                    plans_1 = [elutq.elutq_chain_plan([(l["X"], clones[s_ * n_in], Ys[0], c.N, c.K)]) for s_ in range(n_plans)]
 
-                    def time_chain(plan, n):
-                        for _ in range(3):
-                            elutq.elutq_chain_run(plan, n, stream=stream)
+                    def time_chain(plans, n):
+                        for i_ in range(3):
+                            elutq.elutq_chain_run(plans[i_ % len(plans)], n, stream=stream)
                         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                         a0.record(stream)
-                        for _ in range(reps_pc):
-                            elutq.elutq_chain_run(plan, n, stream=stream)
+                        for i_ in range(reps_pc):
+                            elutq.elutq_chain_run(plans[i_ % len(plans)], n, stream=stream)
                         a1.record(stream)
                         stream.synchronize()
                         return a0.elapsed_time(a1) * 1e3 / reps_pc
 
-                    us_c = max(time_chain(plan_n, n_in) - time_chain(plan_1, 1), 0.0) / (n_in - 1)
+                    us_c = max(time_chain(plans_n, n_in) - time_chain(plans_1, 1), 0.0) / (n_in - 1)
                     per_call[-1].update({"us_in_chain": round(us_c, 3),
                                          "frac_of_hbm_peak_in_chain": round(b / max(us_c, 1e-3) / 1e3 / peak, 3),
-                                         "how_in_chain": "(chain of 9 copies of the layer - chain of 1) / 8, elutq_chain_run"})
-                    if elutq.elutq_chain_status(plan_n) or elutq.elutq_chain_status(plan_1):
-                        per_call[-1]["in_chain_device_status"] = [elutq.elutq_chain_status(plan_n), elutq.elutq_chain_status(plan_1)]
-                    elutq.elutq_chain_forget(plan_n)
-                    elutq.elutq_chain_forget(plan_1)
-                    for cl in clones[1:]:
+                                         "how_in_chain": f"(chain of 9 copies of the layer - chain of 1) / 8, elutq_chain_run, "
+                                                         f"launches rotating over {n_plans} sets of distinct blobs"})
+                    st_ = [elutq.elutq_chain_status(pl) for pl in plans_n + plans_1]
+                    if any(st_):
+                        per_call[-1]["in_chain_device_status"] = [x_ for x_ in st_ if x_]
+                    for pl in plans_n + plans_1:
+                        elutq.elutq_chain_forget(pl)
+                    for cl in clones:
                         elutq.elutq_forget(cl)
-                    del clones, Ys, plan_n, plan_1
+                    del clones, Ys, plans_n, plans_1
                 elutq.elutq_forget(clone)
                 del g2, clone, Y2
 
