@@ -1,5 +1,5 @@
 """Parity at the benchmark's full sizes, in the launch configurations bench.py times (C-ABI calls on a stream with
-library-owned scratch, and the chained decode entry): every call of configs 0, 1, 2, 3 and 4a, and two layers of the
+library-owned scratch, and the chained decode entry): every call of configs 0, 1, 2, 3 and 4a, the whole config-1 and config-3 steps as one plan each, and two layers of the
 32-layer stack of config 4b with their own seeds.  The 8B shapes at M = 1 are compared in full against the fp64
 oracle; the larger problems on a seeded sample of output rows (first and last tiles plus random rows) x all tokens,
 which the oracle computes row by row.  Every comparison is a relative Frobenius error AND an element-wise bound.
@@ -146,6 +146,57 @@ def test_config1_step_through_the_chain_entry(q):
         y = Y[i].cpu().numpy()
         assert hlq.rel_fro_error(y, ref) <= TOL_F16, c
         assert_elementwise(y, ref, hlq.magnitude_bound(Xs[i], layers[i].scales, layers[i].offsets, c.G), c.q, c.K, False, True, c.name)
+    elutq.elutq_chain_forget(plan)
+
+
+def test_config1_whole_step_as_one_plan():
+    """The benchmark's headline launch configuration: all twelve calls in one plan, which elutq_chain_run turns
+    into one launch per bit-width; run three times (epochs), every output compared in full."""
+    calls = workloads.config1_calls()
+    layers = [workloads.hlq_layer(0, c.tag, c.q, c.G, c.N, c.K) for c in calls]
+    packed = [pack_layer(l) for l in layers]
+    Xs = [synth.activations(0, c.tag + "/x", 1, c.K) for c in calls]
+    xd = [x_dev(x) for x in Xs]
+    Y = [torch.zeros((1, c.N), dtype=torch.float16, device="cuda") for c in calls]
+    plan = elutq.elutq_chain_plan([(xd[i], packed[i], Y[i], c.N, c.K) for i, c in enumerate(calls)])
+    for _ in range(3):
+        for y in Y:
+            y.fill_(float("nan"))
+        elutq.elutq_chain_run(plan, len(calls))
+    assert elutq.elutq_chain_status(plan) == 0
+    for i, c in enumerate(calls):
+        ref = hlq.matmul(Xs[i], layers[i].planes, layers[i].scales, layers[i].offsets, c.G)
+        y = Y[i].cpu().numpy()
+        assert np.all(np.isfinite(y)), c
+        assert hlq.rel_fro_error(y, ref) <= TOL_F16, c
+        assert_elementwise(y, ref, hlq.magnitude_bound(Xs[i], layers[i].scales, layers[i].offsets, c.G), c.q, c.K, False, True,
+                           f"{c.name} q{c.q} in the twelve-call plan")
+    elutq.elutq_chain_forget(plan)
+
+
+def test_config3_step_through_the_chain_entry():
+    """The eight 70B calls as one plan (two launches): sampled rows against the oracle, every output finite."""
+    calls = workloads.config3_calls()
+    packed, xd, Y, refs = [], [], [], []
+    for c in calls:
+        layer = workloads.hlq_layer(0, c.tag, c.q, c.G, c.N, c.K)
+        X = synth.activations(0, c.tag + "/x", 1, c.K)
+        rows = _sample_rows(c.N, 512, 8)
+        refs.append((rows, hlq.matmul(X, layer.planes[:, rows], layer.scales[rows], layer.offsets[rows], c.G),
+                     hlq.magnitude_bound(X, layer.scales[rows], layer.offsets[rows], c.G)))
+        packed.append(pack_layer(layer))
+        xd.append(x_dev(X))
+        Y.append(torch.full((1, c.N), float("nan"), dtype=torch.float16, device="cuda"))
+        del layer
+    plan = elutq.elutq_chain_plan([(xd[i], packed[i], Y[i], c.N, c.K) for i, c in enumerate(calls)])
+    elutq.elutq_chain_run(plan, len(calls))
+    assert elutq.elutq_chain_status(plan) == 0
+    for i, c in enumerate(calls):
+        rows, ref, A = refs[i]
+        y = Y[i].cpu().numpy()
+        assert np.all(np.isfinite(y)), c
+        assert hlq.rel_fro_error(y[:, rows], ref) <= TOL_F16, c
+        assert_elementwise(y[:, rows], ref, A, c.q, c.K, False, True, f"config 3 {c.name} q{c.q} in the chain")
     elutq.elutq_chain_forget(plan)
 
 
