@@ -572,7 +572,29 @@ def run_cuda(args) -> None:
     # ---- end to end through the host entry point ---------------------------------------------
     # (a CUDA graph of the public host-buffer calls, whose copy nodes read the pinned inputs and write the pinned
     #  outputs on every replay)
+    host_chain = None
+    if use_chain:
+        # The chained step with host buffers: every call's X in one pinned host arena and every Y in another, one
+        # copy in, the chain's launches, one copy out (elutq_chain_run_host).
+        x_off, y_off = [0], [0]
+        for l in layers:
+            c = l["call"]
+            x_off.append(x_off[-1] + (c.K + 127) // 128 * 128)
+            y_off.append(y_off[-1] + (c.N + 127) // 128 * 128)
+        xh_arena = torch.zeros(x_off[-1], dtype=torch.float16).pin_memory()
+        yh_arena = torch.zeros(y_off[-1], dtype=torch.float16).pin_memory()
+        for i, l in enumerate(layers):
+            xh_arena[x_off[i]:x_off[i] + l["call"].K] = l["Xh"].reshape(-1)
+        xd_arena = torch.zeros(x_off[-1], dtype=torch.float16, device="cuda")
+        yd_arena = torch.zeros(y_off[-1], dtype=torch.float16, device="cuda")
+        plan_h = elutq.elutq_chain_plan([(xd_arena[x_off[i]:], l["packed"], yd_arena[y_off[i]:], l["call"].N, l["call"].K)
+                                         for i, l in enumerate(layers)])
+        host_chain = {"plan": plan_h, "h2d": xh_arena.numel() * 2, "d2h": yh_arena.numel() * 2}
+
     def step_host():
+        if host_chain is not None:
+            elutq.elutq_chain_run_host(host_chain["plan"], len(layers), xd_arena, xh_arena, yd_arena, yh_arena, stream=stream)
+            return
         for l in layers:
             c = l["call"]
             elutq.elutq_lut_gemm_host(l["Xh"], l["packed"], l["Yh"], c.M, c.N, c.K, stream=stream)
@@ -582,7 +604,7 @@ def run_cuda(args) -> None:
         step_host()
         stream.synchronize()
         host_graph = None
-        if not args.no_graph:
+        if not args.no_graph and host_chain is None:
             host_graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(host_graph, stream=stream):
                 step_host()
@@ -603,6 +625,15 @@ def run_cuda(args) -> None:
         h1.record(stream)
         barrier()
         ms_host = h0.elapsed_time(h1)
+        host_chain_bytes, e2e_how = None, "elutq_lut_gemm_host per call (pinned host X in, Y out), CUDA graph"
+        if host_chain is not None:
+            host_chain_bytes = (host_chain["h2d"], host_chain["d2h"])
+            e2e_how = ("elutq_chain_run_host: one copy of the pinned host arena of all X in, the chain's launches, one copy "
+                       "of all Y out to a pinned host arena, per step")
+            e2e_status = elutq.elutq_chain_status(host_chain["plan"], stream=stream)
+            if e2e_status:
+                e2e_how += f"; DEVICE STATUS {e2e_status:#x}"
+            elutq.elutq_chain_forget(host_chain["plan"])
 
         # ---- per-call times: marginal device time of one extra call inside the graph-replayed step -------
         # (the extra call reads its own copy of the packed layer, so it is HBM-cold like the others and
@@ -758,9 +789,9 @@ def run_cuda(args) -> None:
                    "parallelism": "replicas only (independent batch per rank, no collective)"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT,
-                "h2d_bytes_per_step": sum(2 * c.M * c.K for c in calls),
-                "d2h_bytes_per_step": sum(2 * c.M * c.N for c in calls),
-                "how": "elutq_lut_gemm_host per call (pinned host X in, Y out), CUDA graph"},
+                "h2d_bytes_per_step": host_chain_bytes[0] if host_chain_bytes else sum(2 * c.M * c.K for c in calls),
+                "d2h_bytes_per_step": host_chain_bytes[1] if host_chain_bytes else sum(2 * c.M * c.N for c in calls),
+                "how": e2e_how},
         "gpu_launches": launches,
         "clocks": clocks,
         "cpu_baseline": cpu,

@@ -278,13 +278,24 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  *                           Pointers and shapes are frozen in the plan; the buffers they name may change
  *                           content between runs.  M is 1; flags per call: ELUTQ_FLAG_OUT_F32,
  *                           ELUTQ_FLAG_ACCUMULATE (others: ELUTQ_ERR_UNSUPPORTED).
- *   elutq_chain_run         one cooperative launch on `stream` (one CTA per SM; the device must be able to
- *                           hold them all at once, else ELUTQ_ERR_CUDA and nothing runs).  Allocates
- *                           nothing.  Runs of one plan must not overlap on the GPU.  Every CTA first
- *                           compares each blob's header with the plan; on a mismatch the launch ends at
- *                           once with status 0x7C0B and no tile is read.
+ *   elutq_chain_run         one launch on `stream` per run of equal (q, G) (one CTA per SM; the first launch is
+ *                           cooperative: the device must be able to hold its CTAs all at once, else
+ *                           ELUTQ_ERR_CUDA and nothing runs).  Allocates nothing.  Runs of one plan must not
+ *                           overlap on the GPU.  Every CTA first compares the header of each blob of its launch
+ *                           with the plan; on a mismatch that launch ends with status 0x7C0B without reading a
+ *                           tile or writing an output.
  *   elutq_chain_run_opts    the same with an explicit poll limit for the hand-over waits (0 = default, 2^22);
  *                           a test entry.
+ *   elutq_chain_run_host    a run whose activations come from and whose outputs go to HOST memory, with one
+ *                           transfer per direction: on `stream`, copies x_bytes from x_host to x_dev, runs the
+ *                           plan, copies y_bytes from y_dev to y_host.  x_dev and y_dev are the caller's device
+ *                           buffers that the plan's calls point into (typically one arena that holds every
+ *                           call's X and one that holds every Y); x_host and y_host should be pinned, otherwise
+ *                           the copies are synchronous.  A size of 0 skips that copy.  Returns as elutq_chain_run
+ *                           (ELUTQ_ERR_INVALID_ARG for a null pointer with a non-zero size); the outputs are valid
+ *                           on the host when `stream` has been synchronised.  The paper's decode loop keeps
+ *                           activations on the device and has no counterpart of this call; it is the end-to-end
+ *                           form of a step for a caller whose activations live on the host.
  *   elutq_chain_status      synchronises `stream` and reads the plan's status word: 0, or 0x7C05 after a
  *                           hand-over wait ran out (every wait is a bounded poll; the launch then finishes
  *                           without waiting any further and its results are undefined), or 0x7C0B.  After a
@@ -304,6 +315,8 @@ int elutq_chain_plan_bytes(const elutq_gemv_call* calls, int n_calls, size_t* by
 int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size_t plan_bytes, void* stream);
 int elutq_chain_run(void* plan, int n_calls, void* stream);
 int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* stream);
+int elutq_chain_run_host(void* plan, int n_calls, void* x_dev, const void* x_host, size_t x_bytes, const void* y_dev,
+                         void* y_host, size_t y_bytes, void* stream);
 int elutq_chain_status(const void* plan, void* stream, int* status);
 /* The library keeps a small host-side note per planned buffer (which runs of equal (q, G) to launch);
  * elutq_chain_run returns ELUTQ_ERR_SHAPE for a buffer that this process has not planned.  Call this before

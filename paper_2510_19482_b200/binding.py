@@ -59,6 +59,7 @@ _SIGNATURES = {
     "elutq_chain_plan": (c_int, [ctypes.POINTER(GemvCall), c_int, c_void_p, c_size_t, c_void_p]),
     "elutq_chain_run": (c_int, [c_void_p, c_int, c_void_p]),
     "elutq_chain_run_opts": (c_int, [c_void_p, c_int, c_uint, c_void_p]),
+    "elutq_chain_run_host": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_size_t, c_void_p]),
     "elutq_chain_status": (c_int, [c_void_p, c_void_p, ctypes.POINTER(c_int)]),
     "elutq_chain_forget": (c_int, [c_void_p]),
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
@@ -246,6 +247,13 @@ def elutq_chain_run(plan, n_calls: int, stream=None) -> None:
 
 def elutq_chain_run_opts(plan, n_calls: int, wait_limit: int = 0, stream=None) -> None:
     _check(lib().elutq_chain_run_opts(_ptr(plan), n_calls, wait_limit, _stream(stream)), "elutq_chain_run_opts")
+
+
+def elutq_chain_run_host(plan, n_calls: int, x_dev, x_host, y_dev, y_host, stream=None) -> None:
+    """x_host -> x_dev, the plan's launches, y_dev -> y_host, all on `stream` (whole tensors are copied)."""
+    _check(lib().elutq_chain_run_host(_ptr(plan), n_calls, _ptr(x_dev), _ptr(x_host), x_host.numel() * x_host.element_size(),
+                                      _ptr(y_dev), _ptr(y_host), y_host.numel() * y_host.element_size(), _stream(stream)),
+           "elutq_chain_run_host")
 
 
 def elutq_chain_status(plan, stream=None) -> int:

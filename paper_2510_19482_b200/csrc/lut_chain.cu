@@ -1002,6 +1002,22 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* str
     return ELUTQ_OK;
 }
 
+int elutq_chain_run_host(void* plan, int n_calls, void* x_dev, const void* x_host, size_t x_bytes, const void* y_dev,
+                         void* y_host, size_t y_bytes, void* stream) {
+    if ((x_bytes && (!x_dev || !x_host)) || (y_bytes && (!y_dev || !y_host))) return ELUTQ_ERR_INVALID_ARG;
+    if (x_bytes) {
+        const cudaError_t e = cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream);
+        if (e != cudaSuccess) return note_cuda_error((int)e);
+    }
+    const int rc = elutq_chain_run_opts(plan, n_calls, 0, stream);
+    if (rc != ELUTQ_OK) return rc;
+    if (y_bytes) {
+        const cudaError_t e = cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+        if (e != cudaSuccess) return note_cuda_error((int)e);
+    }
+    return ELUTQ_OK;
+}
+
 int elutq_chain_run(void* plan, int n_calls, void* stream) {
     return elutq_chain_run_opts(plan, n_calls, 0u, stream);
 }

@@ -123,6 +123,30 @@ def test_chain_accumulate_flag_adds_into_y():
     assert hlq.rel_fro_error(Y.cpu().numpy(), ref) <= TOL_F32
 
 
+def test_chain_with_host_buffers_moves_one_arena_per_direction():
+    # every call's X in one pinned host arena, every Y in another: one copy in, the launches, one copy out
+    shapes = [(2, 128, 300, 1024), (3, 128, 128, 2048), (2, 64, 77, 512)]
+    layers, Xs = _build(shapes, 27, "chain-host")
+    packed = [pack_layer(l) for l in layers]
+    x_off = np.cumsum([0] + [l.K for l in layers])                     # in fp16 elements; K is a multiple of 32
+    y_off = np.cumsum([0] + [(l.N + 127) // 128 * 128 for l in layers])
+    x_host = torch.empty(int(x_off[-1]), dtype=torch.float16).pin_memory()
+    y_host = torch.full((int(y_off[-1]),), float("nan"), dtype=torch.float16).pin_memory()
+    for i, X in enumerate(Xs):
+        x_host[int(x_off[i]):int(x_off[i + 1])] = torch.from_numpy(X.view(np.int16)).view(torch.float16).reshape(-1)
+    x_dev = torch.zeros_like(x_host, device="cuda")
+    y_dev = torch.zeros_like(y_host, device="cuda")
+    calls = [(x_dev[int(x_off[i]):], packed[i], y_dev[int(y_off[i]):], l.N, l.K) for i, l in enumerate(layers)]
+    plan = elutq.elutq_chain_plan(calls)
+    elutq.elutq_chain_run_host(plan, len(calls), x_dev, x_host, y_dev, y_host)
+    assert elutq.elutq_chain_status(plan) == 0          # (synchronises the stream)
+    for i, l in enumerate(layers):
+        ref = hlq.matmul(Xs[i], l.planes, l.scales, l.offsets, l.G)
+        y = y_host[int(y_off[i]):int(y_off[i]) + l.N].numpy().reshape(1, -1)
+        assert hlq.rel_fro_error(y, ref) <= TOL_F16, shapes[i]
+    elutq.elutq_chain_forget(plan)
+
+
 def test_a_hand_over_wait_that_runs_out_ends_the_launch_with_a_status():
     # Call 1 reads what call 0 writes, so it waits for call 0's completion count.  Call 0 is planned with the
     # test-only flag that leaves out its completion signal and the poll limit is set to 4096: the wait runs out,
