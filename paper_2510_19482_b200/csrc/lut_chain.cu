@@ -492,9 +492,9 @@ struct ChainCtx {
 __device__ __forceinline__ void desc_fetch(const ChainCtx& x, int slot_warp, int c, int lane) {
     if (lane < 9 && c < x.c_end) slot_fetch(warp_slot(slot_warp, c), x.calls, x.parts, x.grid, c, lane);
 }
-__device__ __forceinline__ void desc_begin(const ChainCtx& x, int slot_warp, int lane) {
-    desc_fetch(x, slot_warp, x.c_begin, lane);
-    desc_fetch(x, slot_warp, x.c_begin + 1, lane);
+__device__ __forceinline__ void desc_begin(const ChainCtx& x, int slot_warp, int c0, int lane) {
+    desc_fetch(x, slot_warp, c0, lane);
+    desc_fetch(x, slot_warp, c0 + 1, lane);
     if (lane < 9) cp_async_wait_all();
     __syncwarp();
 }
@@ -751,8 +751,12 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         // K-split reduction of every call this CTA works on, then the call's completion report
         const int fw = warp - kLookupWarps - kBuilderWarps, ft = tid - (kLookupWarps + kBuilderWarps) * 32;
         unsigned phases = 0;                  // parities of this warp's copy barriers
-        desc_begin(x, fw, lane);
-        for (int c = c_begin; c < c_end; ++c) {
+        // The reduction of a launch's last call is left to the finishers of the chain's next launch (their CTAs
+        // move in as this launch's leave): otherwise every CTA of this launch would stay until its finishers have
+        // fetched the last partial sums, a copy round trip after the last look-up, with the rest of the SM idle.
+        const int f_begin = first_run ? c_begin : c_begin - 1, f_end = last_run ? c_end : c_end - 1;
+        desc_begin(x, fw, f_begin, lane);
+        for (int c = f_begin; c < f_end; ++c) {
             const ChainSlot* sl = desc_next(x, fw, c, lane);
             const ChainCall* d = &sl->d;
             if (bid < d->n_ctas && d->n_kc > 1) {
