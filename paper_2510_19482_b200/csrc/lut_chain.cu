@@ -20,7 +20,9 @@
 //     one bulk copy (two copies in flight per warp, completion on an mbarrier), adds the chunks in ascending order -
 //     bit-reproducible -, checks the tags, repeats the copy (bounded) while a tag is not this call's yet, writes Y
 //     and reports the call's completion on a counter.  No fence, no ticket, no second kernel for the reduction: the
-//     copy that finds the tags is the copy that brings the values.
+//     copy that finds the tags is the copy that brings the values.  (The last call of a launch that another
+//     launch of the chain follows is reduced by that launch's finishers, so that the CTAs leave right after their
+//     last look-up.)
 //   * Ordering: the result is what the calls give when run one after another.  The plan records, from the buffer
 //     addresses, which earlier calls a call really depends on (its X or Y overlaps their Y, or its Y their X);
 //     before the builders read X they wait (bounded) for the completion counters of exactly those calls.  Calls
