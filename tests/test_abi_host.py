@@ -101,6 +101,10 @@ def test_chain_argument_validation_happens_on_the_host():
     assert L.elutq_chain_run(None, 2, None) == -1
     assert L.elutq_chain_run(256, 2, None) == -2                              # a buffer that was never planned
     assert L.elutq_chain_status(None, None, None) == -1
+    # the host-buffer form: a null pointer with a non-zero size is refused before anything is copied or launched
+    assert L.elutq_chain_run_host(256, 2, None, 4096, 64, 512, 8192, 64, None) == -1
+    assert L.elutq_chain_run_host(256, 2, 512, 4096, 64, 512, None, 64, None) == -1
+    assert L.elutq_chain_run_host(256, 2, None, None, 0, None, None, 0, None) == -2      # no copies asked for: a plain run of an unplanned buffer
     assert L.elutq_reserve(0, 16, 512, None) == -1
     assert L.elutq_scratch_address(None, 9, None, None) == -1
     assert elutq.elutq_launch_count() == before
