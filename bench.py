@@ -574,8 +574,8 @@ def run_cuda(args) -> None:
     #  outputs on every replay)
     host_chain = None
     if use_chain:
-        # The chained step with host buffers: every call's X in one pinned host arena and every Y in another, one
-        # copy in, the chain's launches, one copy out (elutq_chain_run_host).
+        # The chained step with host buffers: every call's X in one pinned host arena and every Y in another; a step
+        # is one copy in and the chain's launches (elutq_chain_run_host), which write Y into the host arena.
         x_off, y_off = [0], [0]
         for l in layers:
             c = l["call"]
@@ -586,14 +586,14 @@ def run_cuda(args) -> None:
         for i, l in enumerate(layers):
             xh_arena[x_off[i]:x_off[i] + l["call"].K] = l["Xh"].reshape(-1)
         xd_arena = torch.zeros(x_off[-1], dtype=torch.float16, device="cuda")
-        yd_arena = torch.zeros(y_off[-1], dtype=torch.float16, device="cuda")
-        plan_h = elutq.elutq_chain_plan([(xd_arena[x_off[i]:], l["packed"], yd_arena[y_off[i]:], l["call"].N, l["call"].K)
+        # the calls' Y point into the pinned host arena: the reduction's stores cross the bus during the launch
+        plan_h = elutq.elutq_chain_plan([(xd_arena[x_off[i]:], l["packed"], yh_arena[y_off[i]:], l["call"].N, l["call"].K)
                                          for i, l in enumerate(layers)])
-        host_chain = {"plan": plan_h, "h2d": xh_arena.numel() * 2, "d2h": yh_arena.numel() * 2}
+        host_chain = {"plan": plan_h, "h2d": xh_arena.numel() * 2, "d2h": sum(2 * l["call"].N for l in layers)}
 
     def step_host():
         if host_chain is not None:
-            elutq.elutq_chain_run_host(host_chain["plan"], len(layers), xd_arena, xh_arena, yd_arena, yh_arena, stream=stream)
+            elutq.elutq_chain_run_host(host_chain["plan"], len(layers), xd_arena, xh_arena, stream=stream)
             return
         for l in layers:
             c = l["call"]
@@ -628,8 +628,8 @@ def run_cuda(args) -> None:
         host_chain_bytes, e2e_how = None, "elutq_lut_gemm_host per call (pinned host X in, Y out), CUDA graph"
         if host_chain is not None:
             host_chain_bytes = (host_chain["h2d"], host_chain["d2h"])
-            e2e_how = ("elutq_chain_run_host: one copy of the pinned host arena of all X in, the chain's launches, one copy "
-                       "of all Y out to a pinned host arena, per step")
+            e2e_how = ("elutq_chain_run_host: one copy of the pinned host arena of all X in, then the chain's launches, whose "
+                       "calls have their Y in a pinned host arena (the reduction stores straight into host memory), per step")
             e2e_status = elutq.elutq_chain_status(host_chain["plan"], stream=stream)
             if e2e_status:
                 e2e_how += f"; DEVICE STATUS {e2e_status:#x}"

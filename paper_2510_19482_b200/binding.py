@@ -249,11 +249,13 @@ def elutq_chain_run_opts(plan, n_calls: int, wait_limit: int = 0, stream=None) -
     _check(lib().elutq_chain_run_opts(_ptr(plan), n_calls, wait_limit, _stream(stream)), "elutq_chain_run_opts")
 
 
-def elutq_chain_run_host(plan, n_calls: int, x_dev, x_host, y_dev, y_host, stream=None) -> None:
-    """x_host -> x_dev, the plan's launches, y_dev -> y_host, all on `stream` (whole tensors are copied)."""
-    _check(lib().elutq_chain_run_host(_ptr(plan), n_calls, _ptr(x_dev), _ptr(x_host), x_host.numel() * x_host.element_size(),
-                                      _ptr(y_dev), _ptr(y_host), y_host.numel() * y_host.element_size(), _stream(stream)),
-           "elutq_chain_run_host")
+def elutq_chain_run_host(plan, n_calls: int, x_dev, x_host, y_dev=None, y_host=None, stream=None) -> None:
+    """x_host -> x_dev, the plan's launches, y_dev -> y_host, all on `stream` (whole tensors are copied; a pair that
+    is None is not copied: e.g. when the plan's Y pointers name pinned host memory themselves)."""
+    xb = 0 if x_host is None else x_host.numel() * x_host.element_size()
+    yb = 0 if y_host is None else y_host.numel() * y_host.element_size()
+    _check(lib().elutq_chain_run_host(_ptr(plan), n_calls, _ptr(x_dev), _ptr(x_host), xb, _ptr(y_dev), _ptr(y_host), yb,
+                                      _stream(stream)), "elutq_chain_run_host")
 
 
 def elutq_chain_status(plan, stream=None) -> int:

@@ -144,7 +144,16 @@ def test_chain_with_host_buffers_moves_one_arena_per_direction():
         ref = hlq.matmul(Xs[i], l.planes, l.scales, l.offsets, l.G)
         y = y_host[int(y_off[i]):int(y_off[i]) + l.N].numpy().reshape(1, -1)
         assert hlq.rel_fro_error(y, ref) <= TOL_F16, shapes[i]
+    # the same with the calls' Y in pinned host memory themselves: no copy out, bit-identical outputs
+    y_host2 = torch.full((int(y_off[-1]),), float("nan"), dtype=torch.float16).pin_memory()
+    plan2 = elutq.elutq_chain_plan([(x_dev[int(x_off[i]):], packed[i], y_host2[int(y_off[i]):], l.N, l.K) for i, l in enumerate(layers)])
+    elutq.elutq_chain_run_host(plan2, len(calls), x_dev, x_host)
+    assert elutq.elutq_chain_status(plan2) == 0
+    for i, l in enumerate(layers):
+        a, b = int(y_off[i]), int(y_off[i]) + l.N
+        assert torch.equal(y_host2[a:b].view(torch.int16), y_host[a:b].view(torch.int16)), shapes[i]
     elutq.elutq_chain_forget(plan)
+    elutq.elutq_chain_forget(plan2)
 
 
 def test_a_hand_over_wait_that_runs_out_ends_the_launch_with_a_status():
