@@ -42,7 +42,7 @@ namespace elutq {
 namespace {
 
 constexpr unsigned kChainMagic = 0x4E494843u;
-constexpr int kChainRegions = 3;              // scratch regions for the tagged partial sums, used round-robin
+constexpr int kChainRegions = 6;              // scratch regions for the tagged partial sums, used round-robin
 constexpr int kDescSlots = 4;
 constexpr int kLookupWarps = 26;              // (22 or 18 look-up warps with 72 / 80 registers each measured slower)
 constexpr int kBuilderWarps = 4;
@@ -283,8 +283,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity) {     
 // long as its look-ups on every shape with more than a few row blocks per CTA.  `phases` holds the barrier parities
 // of the warp's slots across calls.  Bounded: `limit` sweeps over the ring without a complete copy end the launch
 // with the wait-expired status.
+// `first_issued`: the warp's first copies of this call (slot k: block k) are in flight already, see chain_reduce_ahead.
 __device__ __noinline__ unsigned chain_reduce(const ChainCall* d, const ChainPart p, unsigned tag, unsigned limit,
-                                              unsigned* status, int fw, int lane, unsigned phases) {
+                                              unsigned* status, int fw, int lane, unsigned phases, bool first_issued) {
     ChainShared* sh = chain_shared();
     const int n_kc = d->n_kc, N = d->N, groups = d->groups;
     constexpr int D = kFinSlots;                               // ring slots in use
@@ -310,8 +311,12 @@ __device__ __noinline__ unsigned chain_reduce(const ChainCall* d, const ChainPar
         seg[k] = 0; sums[k] = 0.f;
     }
 #pragma unroll
-    for (int k = 0; k < kFinSlots; ++k)
-        if (blk[k] < nblk) issue(k, blk[k], 0);
+    for (int k = 0; k < kFinSlots; ++k) {
+        if (blk[k] < nblk) {
+            if (first_issued) pending |= 1u << k;
+            else issue(k, blk[k], 0);
+        }
+    }
     int remaining = nblk;
     unsigned idle = 0;
     while (remaining > 0) {
@@ -377,6 +382,28 @@ __device__ __noinline__ unsigned chain_reduce(const ChainCall* d, const ChainPar
         }
     }
     return phases;
+}
+
+// The warp's first copies of a call, issued before the call before it is reported complete: the report is a release
+// (it holds the reporting thread until the call's outputs have reached memory), and with the next call's first copies
+// already under way that round trip and theirs overlap instead of following one another (measured with the release
+// taken out: 3 - 9 us on a sixteen-call chain of one 8B layer).  All of the warp's ring slots are free at that point.
+__device__ __forceinline__ void chain_reduce_ahead(const ChainCall* d, const ChainPart p, int fw, int lane) {
+    const int n_kc = d->n_kc, groups = d->groups;
+    constexpr int buf_bytes = kFinRingBytes / kFinSlots;
+    const int first = p.rb0 + p.grp + fw * groups;
+    const int nblk = first < p.rb1 ? (p.rb1 - first + kFinisherWarps * groups - 1) / (kFinisherWarps * groups) : 0;
+    uint8_t* const ring = chain_smem + kOffFinBuf + fw * kFinRingBytes;
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < kFinSlots; ++k) {
+            if (k < nblk) {
+                const int rb = first + k * kFinisherWarps * groups;
+                fin_copy(ring + k * buf_bytes, d->slots + (size_t)rb * n_kc * kTileRows, (unsigned)min(32, n_kc) * kTileRows * 8,
+                         fin_bar(fw, k));
+            }
+        }
+    }
 }
 
 // The lane's 16 activations of chunk kc (two byte-columns), as (x_i of column 2*lane, x_i of column 2*lane+1).
@@ -758,17 +785,29 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         // fetched the last partial sums, a copy round trip after the last look-up, with the rest of the SM idle.
         const int f_begin = first_run ? c_begin : c_begin - 1, f_end = last_run ? c_end : c_end - 1;
         desc_begin(x, fw, f_begin, lane);
+        const ChainSlot* sl = f_begin < f_end ? desc_next(x, fw, f_begin, lane) : nullptr;
+        bool first_issued = false;            // this call's first copies were issued during the call before
         for (int c = f_begin; c < f_end; ++c) {
-            const ChainSlot* sl = desc_next(x, fw, c, lane);
             const ChainCall* d = &sl->d;
-            if (bid < d->n_ctas && d->n_kc > 1) {
-                const ChainPart p = chain_part(sl);
+            const bool mine = bid < d->n_ctas && d->n_kc > 1;
+            const unsigned flags = d->flags;
+            if (mine) {
                 const unsigned tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
-                phases = chain_reduce(d, p, tag, spin_limit, status, fw, lane, phases);
+                phases = chain_reduce(d, chain_part(sl), tag, spin_limit, status, fw, lane, phases, first_issued);
+            }
+            // the next call's descriptor (requested two calls ago), and its first copies before this call's report
+            const ChainSlot* sl_next = c + 1 < f_end ? desc_next(x, fw, c + 1, lane) : nullptr;
+            first_issued = false;
+            if (sl_next != nullptr && bid < sl_next->d.n_ctas && sl_next->d.n_kc > 1 && !sh->abort) {
+                chain_reduce_ahead(&sl_next->d, chain_part(sl_next), fw, lane);
+                first_issued = true;
+            }
+            if (mine) {
                 bar_finishers();              // every row of this CTA is stored
-                if (ft == 0 && !(d->flags & kCallTestNoSignal)) red_release_add(done + c, 1u);
+                if (ft == 0 && !(flags & kCallTestNoSignal)) red_release_add(done + c, 1u);
             }
             __syncwarp();
+            sl = sl_next;
         }
     }
 }
