@@ -7,8 +7,9 @@
 // model has one such pair, so normally the whole list is one launch; a list that mixes them is cut into one
 // launch per run.  Inside a CTA the warps are specialised (Appendix B's two phases run side by side):
 //
-//   * 4 builder warps load the activations of the CTA's next K chunk and fill the other of two table buffers
-//     (fused 8-bit tables, 64 KiB each); before they build a job they publish a small record of it (first item,
+//   * 4 builder warps, as two teams of two (team t: the table jobs of parity t, always in table buffer t), load the
+//     activations of the CTA's next K chunk and fill the table buffers (fused 8-bit tables, 64 KiB each); before a
+//     team builds a job it publishes a small record of it (first item,
 //     row-block range, where the partial sums go, tag) in shared memory;
 //   * 26 look-up warps follow those records: they stream the packed weights of the job (one warp per 16-row x
 //     512-column item, registers refilled one item ahead as in lut_gemv.cu, also across job boundaries) and sum table
@@ -46,9 +47,12 @@ constexpr int kChainRegions = 6;              // scratch regions for the tagged 
 constexpr int kDescSlots = 4;
 constexpr int kLookupWarps = 26;              // (22 or 18 look-up warps with 72 / 80 registers each measured slower)
 constexpr int kBuilderWarps = 4;
+constexpr int kTeamWarps = 2;                 // builder warps per team; team t builds table buffer t (the jobs of parity t)
+constexpr int kBuilderTeams = kBuilderWarps / kTeamWarps;
 constexpr int kFinisherWarps = 2;
 constexpr int kChainThreads = (kLookupWarps + kBuilderWarps + kFinisherWarps) * 32;
-constexpr int kBuilderThreads = kBuilderWarps * 32;
+constexpr int kTeamThreads = kTeamWarps * 32;
+static_assert(kBuilderTeams == 2, "one builder team per table buffer");
 constexpr int kFinisherThreads = kFinisherWarps * 32;
 // shared memory: two table buffers, then per buffer 16 group sums, four mbarriers, flags, descriptor ring
 constexpr int kOffGsum = 2 * kTableBytes;
@@ -56,11 +60,11 @@ constexpr int kOffBar = kOffGsum + 128;
 constexpr int kOffShared = kOffBar + 32;
 constexpr int kOffRecBar = kOffGsum + 192;                // one "record written" barrier per job record
 constexpr int kSlotBytes = 144;                           // descriptor (128) + this CTA's share of the call (16)
-constexpr int kOffDesc = kOffGsum + 256;                  // builders' descriptor ring
-constexpr int kOffWarpDesc = kOffDesc + kDescSlots * kSlotBytes;   // finisher warps: a descriptor ring per warp
-constexpr int kOffJobRec = kOffWarpDesc + kFinisherWarps * kDescSlots * kSlotBytes;   // job records, written by the builders
+constexpr int kOffWarpDesc = kOffGsum + 256;              // a descriptor ring per finisher warp and per builder warp
+constexpr int kWarpRings = kFinisherWarps + kBuilderWarps;
+constexpr int kOffJobRec = kOffWarpDesc + kWarpRings * kDescSlots * kSlotBytes;   // job records, written by the builders
 constexpr int kJobRecs = 4;
-static_assert(kOffShared + 32 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffDesc, "shared-memory layout");
+static_assert(kOffShared + 32 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffWarpDesc, "shared-memory layout");
 // finisher warps: a ring of buffers per warp that bulk copies fill with the partial sums of one row block
 constexpr int kFinSlots = 2;                  // copies in flight per finisher warp (measured on the 8B step and the
                                               // 32-layer stack: 1: 77.8 / 562 us, 2: 79.1 / 541 us, 4: 82.7 / 580 us, 8: 88 / 651 us)
@@ -93,7 +97,8 @@ struct ChainCall {                            // 128 bytes
     unsigned done_target;                     // completion reports per launch: one per CTA (one per look-up warp of every
                                               // CTA when the call has no K split)
     int release;                              // 1: a later call of the plan waits for this one (see red_release_add)
-    int pad[6];
+    unsigned guard_target;                    // done_target of call guard_call
+    int pad[5];
 };
 static_assert(sizeof(ChainCall) == 128, "descriptor size");
 static_assert(sizeof(ChainCtl) <= 256, "control block size");
@@ -106,9 +111,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ void prefetch_l2_line(const void* p) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
     const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
@@ -116,8 +118,9 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
 __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
-__device__ __forceinline__ void bar_builders() {          // named barrier 1: the builder warps only
-    asm volatile("bar.sync 1, %0;" ::"n"(kBuilderThreads) : "memory");
+__device__ __forceinline__ void bar_team(int team) {      // named barriers 1 and 4: the warps of one builder team
+    if (team == 0) asm volatile("bar.sync 1, %0;" ::"n"(kTeamThreads) : "memory");
+    else asm volatile("bar.sync 4, %0;" ::"n"(kTeamThreads) : "memory");
 }
 __device__ __forceinline__ void bar_lookups() {           // named barrier 3: the look-up warps only
     asm volatile("bar.sync 3, %0;" ::"n"(kLookupWarps * 32) : "memory");
@@ -143,7 +146,6 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, unsigned parity) {
 struct ChainShared {
     volatile int abort;                       // a wait ran out: stop waiting
     unsigned epoch;
-    volatile unsigned recs_published;         // job records written so far (by the builders)
     volatile int headers_bad;                 // a blob of this launch no longer carries the header it was planned with
 };
 static_assert(sizeof(ChainShared) <= 32, "shared flags");
@@ -178,10 +180,6 @@ struct ChainSlot {                            // what a role keeps of a call in 
     int4 part;                                // this CTA's share: rb0, rb1, kc0, nseg | grp << 16
 };
 static_assert(sizeof(ChainSlot) == kSlotBytes, "slot size");
-__device__ __forceinline__ ChainSlot* chain_slot(int c) {
-    return reinterpret_cast<ChainSlot*>(chain_smem + kOffDesc) + (c & (kDescSlots - 1));
-}
-__device__ __forceinline__ ChainCall* chain_desc(int c) { return &chain_slot(c)->d; }
 __device__ __forceinline__ ChainSlot* warp_slot(int fw, int c) {
     return reinterpret_cast<ChainSlot*>(chain_smem + kOffWarpDesc) + fw * kDescSlots + (c & (kDescSlots - 1));
 }
@@ -451,8 +449,8 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
         A[6] = fadd2(A[2], x[2]);
         A[7] = fadd2(A[3], x[2]);
 #pragma unroll
-        for (int s = 0; s < 16 / kBuilderWarps; ++s) {
-            const int hi = bw + s * kBuilderWarps;
+        for (int s = 0; s < 16 / kTeamWarps; ++s) {
+            const int hi = bw + s * kTeamWarps;
             float2 Bv = make_float2(0.f, 0.f);
 #pragma unroll
             for (int b = 0; b < 4; ++b)
@@ -491,7 +489,7 @@ __device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&co
     for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
         const bool in_job = rb + kLookupWarps < rb1;
         const uint8_t* nvp = vp + kLookupWarps * C::TILE_BYTES;
-        if (!in_job && chain_shared()->recs_published > job + 1) {
+        if (!in_job && __all_sync(0xffffffffu, mbar_test(bar_rec(job + 1), ((job + 1) >> 2) & 1u))) {
             const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
             if ((int)n0.z + lw < (int)n0.w) {
                 nvp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + warp_off;
@@ -617,9 +615,11 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
     // The plan is the one the host launched (its parts are addressed through kernel arguments: no pointer is
     // chased through the control block on the way to the first descriptor).
     const int grid = (int)gridDim.x;
-    if (tid < 16 * min(c_end - c_begin, 3)) {
-        const int c = c_begin + (tid >> 4);
-        slot_fetch(chain_slot(c), calls, parts, grid, c, tid & 15);
+    if (warp >= kLookupWarps && warp < kLookupWarps + kBuilderWarps && lane < 9) {
+        // every builder warp keeps its own copies of the descriptors it works through (no barrier between the teams)
+        const int ring = kFinisherWarps + (warp - kLookupWarps);
+        if (c_begin < c_end) slot_fetch(warp_slot(ring, c_begin), calls, parts, grid, c_begin, lane);
+        if (c_begin + 1 < c_end) slot_fetch(warp_slot(ring, c_begin + 1), calls, parts, grid, c_begin + 1, lane);
     }
     // Header check, first part: the look-up threads 64, 65, ... read the header of one call's blob each.  The loads
     // are issued here and looked at after the barrier below, so that they are on their way while the descriptors
@@ -641,12 +641,11 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         epoch_now = ctl->epoch;
         sh->abort = 0;
         sh->headers_bad = 0;
-        sh->recs_published = 0;
         sh->epoch = epoch_now;
         // one arrival per warp (its lane 0, after the warp has converged): 32 arrivals of a warp on one barrier word
         // would be 32 serialised shared-memory atomics
-        mbar_init(bar_full(0), kBuilderWarps);
-        mbar_init(bar_full(1), kBuilderWarps);
+        mbar_init(bar_full(0), kTeamWarps);
+        mbar_init(bar_full(1), kTeamWarps);
         mbar_init(bar_free(0), kLookupWarps);
         mbar_init(bar_free(1), kLookupWarps);
         for (int j = 0; j < kJobRecs; ++j) mbar_init(bar_rec(j), 1);
@@ -699,47 +698,42 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         }
     } else if (warp < kLookupWarps + kBuilderWarps) {
         // ---------------------------------------------------------------- builder warps
-        const int bw = warp - kLookupWarps, bt = tid - kLookupWarps * 32;
-        unsigned job = 0;
+        // Two teams of two warps; team t builds the jobs of parity t, always into table buffer t, so the per-call
+        // latencies of one team's job (descriptor, activation load, record, waits, hand-over) run beside the other
+        // team's.  Both teams walk every call to count the jobs; a team works on the segments of its parity.
+        const int bw = warp - kLookupWarps, team = bw / kTeamWarps, tw = bw % kTeamWarps;
+        const bool lead = tw == 0 && lane == 0;               // the team's thread for records, waits on counters
+        const int ring = kFinisherWarps + bw;
+        const int b = team;
+        unsigned job = 0;                                     // jobs of this CTA before the current call
         for (int c = c_begin; c < c_end; ++c) {
-            const ChainCall* d = chain_desc(c);
-            // descriptor three calls ahead (its slot was last read one call ago); it is waited for at the end of this
-            // iteration and published by the barrier of the next one
-            if (c + 3 < c_end && bt < 9) slot_fetch(chain_slot(c + 3), calls, parts, grid, c + 3, bt);
+            const ChainSlot* sl = desc_next(x, ring, c, lane);
+            const ChainCall* d = &sl->d;
             const bool work = bid < d->n_ctas;
-            ChainPart p = {0, 0, 0, 0, 0};
-            if (work) {
-                p = chain_part(chain_slot(c));
-            }
-            if (c + 1 < c_end && bt >= 32 && bt < 40) {
-                // activations of the next call's first chunk on this CTA: into L2 ahead of its table build
-                const ChainCall* dn = chain_desc(c + 1);
-                if (bid < dn->n_ctas) {
-                    const int k0 = chain_slot(c + 1)->part.z * kChunkK + (bt - 32) * 64;
-                    if (k0 < dn->K) prefetch_l2_line(dn->X + k0);
+            const ChainPart p = chain_part(sl);
+            const int nseg = work ? p.nseg : 0;
+            const int seg0 = ((job & 1u) == (unsigned)team) ? 0 : 1;      // this team's first segment of the call
+            if (seg0 < nseg) {
+                if (d->dep_first <= d->dep_last) {
+                    // as-if-sequential order: every earlier call whose output this call reads or overwrites (or whose
+                    // input it overwrites) is complete
+                    if (lead && !sh->abort) {
+                        bool ok = true;
+                        for (int j = d->dep_first; ok && j <= d->dep_last; ++j)
+                            ok = wait_reached(done + j, (epoch + 1u) * calls[j].done_target, spin_limit);
+                        if (!ok) raise_abort(status);
+                    }
+                    bar_team(team);
                 }
-            }
-            if (d->dep_first <= d->dep_last) {
-                // as-if-sequential order: every earlier call whose output this call reads or overwrites (or whose
-                // input it overwrites) is complete
-                if (bt == 0 && !sh->abort) {
-                    bool ok = true;
-                    for (int j = d->dep_first; ok && j <= d->dep_last; ++j)
-                        ok = wait_reached(done + j, (epoch + 1u) * calls[j].done_target, spin_limit);
-                    if (!ok) raise_abort(status);
-                }
-                bar_builders();
-            }
-            if (work) {
-                for (int seg = 0; seg < p.nseg; ++seg, ++job) {
-                    const int b = job & 1;
+                for (int seg = seg0; seg < nseg; seg += kBuilderTeams) {
+                    const unsigned j = job + (unsigned)seg;
                     float2 xv[8];             // requested before the wait for the buffer: the load latency overlaps it
                     load_x_pairs(xv, d->X, p.kc0 + seg, d->K, lane);
-                    if (bt == 0) {
+                    if (lead) {
                         // the job's record, published before the tables are built: the look-up warps may already request
                         // their first item of this job while they work on the one before (the record's slot was last
                         // read four jobs ago)
-                        JobRec* r = job_rec(job);
+                        JobRec* r = job_rec(j);
                         const int kc = p.kc0 + seg;
                         r->tile0 = d->tiles + ((size_t)kc * d->n_rb + p.rb0) * Cfg<Q, G>::TILE_BYTES;
                         r->out = d->n_kc > 1 ? d->slots + (size_t)kc * kTileRows : nullptr;
@@ -749,38 +743,33 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
                         r->rb0 = p.rb0; r->rb1 = p.rb1; r->N = d->N;
                         r->flags = d->flags;
                         r->tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
-                        r->last = (seg + 1 == p.nseg ? 1 : 0) | (d->release ? 2 : 0);
+                        r->last = (seg + 1 == nseg ? 1 : 0) | (d->release ? 2 : 0);
                         r->stop = 0;
                         __threadfence_block();
-                        sh->recs_published = job + 1;
-                        mbar_arrive(bar_rec(job));
+                        mbar_arrive(bar_rec(j));
                     }
-                    if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);   // look-ups of job - 2 are over
-                    build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), xv, bw, lane);
-                    if (seg == 0 && d->guard_call >= 0) {
-                        // the scratch region of this call was last used by call guard_call: its reductions must be over
-                        // before the look-up warps store into it (they start when the tables are handed over)
-                        if (bt == 0 && !sh->abort &&
-                            !wait_reached(done + d->guard_call, (epoch + 1u) * calls[d->guard_call].done_target, spin_limit))
-                            raise_abort(status);
-                        bar_builders();
-                    }
+                    if (j >= 2) mbar_wait(bar_free(b), ((j - 2) >> 1) & 1, spin_limit, status);   // look-ups of job j - 2 are over
+                    build_tables_bw<G>(smem + b * kTableBytes, reinterpret_cast<float*>(smem + kOffGsum + b * 64), xv, tw, lane);
+                    // the scratch region of this call was last used by call guard_call: its reductions must be over
+                    // before the look-up warps store into it; they start when the LAST warp of the team hands the tables
+                    // over, so it is enough that the lead waits before its own arrival
+                    if (lead && seg == 0 && d->guard_call >= 0 && !sh->abort &&
+                        !wait_reached(done + d->guard_call, (epoch + 1u) * d->guard_target, spin_limit))
+                        raise_abort(status);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_full(b));
                 }
             }
-            if (bt < 9) cp_async_wait_all();
-            bar_builders();                   // descriptor c + 3 has landed for every builder thread
+            job += (unsigned)nseg;
         }
-        {   // the record that ends the look-up warps' loop, handed over like a job
-            const int b = job & 1;
+        if ((job & 1u) == (unsigned)team) {
+            // the record that ends the look-up warps' loop, handed over like a job (by the team whose turn it is)
             if (job >= 2) mbar_wait(bar_free(b), ((job - 2) >> 1) & 1, spin_limit, status);
-            if (bt == 0) {
+            if (lead) {
                 JobRec* r = job_rec(job);
                 r->rb0 = 0; r->rb1 = 0;
                 r->stop = 1;
                 __threadfence_block();
-                sh->recs_published = job + 1;
                 mbar_arrive(bar_rec(job));
             }
             __syncwarp();
@@ -1010,6 +999,7 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
             pt[b] = v;
         }
         d.guard_call = i >= kChainRegions ? i - kChainRegions : -1;
+        d.guard_target = d.guard_call >= 0 ? dc[d.guard_call].done_target : 0u;
         d.done_target = (unsigned)(g.n_kc > 1 ? d.n_ctas : d.n_ctas * kLookupWarps);
         if (runs.n_runs == 0 || runs.q[runs.n_runs - 1] != q || runs.G[runs.n_runs - 1] != G) {
             if (runs.n_runs == kMaxRuns) return ELUTQ_ERR_UNSUPPORTED;
