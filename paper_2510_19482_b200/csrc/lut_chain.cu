@@ -522,23 +522,25 @@ struct ChainCtx {
     unsigned epoch, spin_limit;
 };
 
-// Per-warp descriptor copies for the warps that run on their own (look-up and finisher warps): the copies of
-// calls c + 1 and c + 2 are on their way or there while call c is worked on.
+// Per-warp descriptor copies for the warps that walk the calls on their own (builder and finisher warps): a ring of
+// four slots, filled by asynchronous copies two calls ahead, one copy group per call.  Taking call c waits only for
+// the groups before the newest one, so the copy of call c + 1 may still be in flight: a walk that waited for it too
+// was bound by one global round trip per call (0.9 us, measured on a chain of small calls with everything else off).
 __device__ __forceinline__ void desc_fetch(const ChainCtx& x, int slot_warp, int c, int lane) {
-    if (lane < 9 && c < x.c_end) slot_fetch(warp_slot(slot_warp, c), x.calls, x.parts, x.grid, c, lane);
+    if (lane < 9) {
+        if (c < x.c_end) slot_fetch(warp_slot(slot_warp, c), x.calls, x.parts, x.grid, c, lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");      // (an empty group past the end keeps the count)
+    }
 }
 __device__ __forceinline__ void desc_begin(const ChainCtx& x, int slot_warp, int c0, int lane) {
     desc_fetch(x, slot_warp, c0, lane);
     desc_fetch(x, slot_warp, c0 + 1, lane);
-    if (lane < 9) cp_async_wait_all();
-    __syncwarp();
 }
-// descriptor of call c for this warp; call c + 1 has landed too, call c + 2 is requested
+// descriptor of call c for this warp; call c + 1 is on its way or there, call c + 2 is requested
 __device__ __forceinline__ const ChainSlot* desc_next(const ChainCtx& x, int slot_warp, int c, int lane) {
-    if (lane < 9) cp_async_wait_all();            // c + 1 (requested one call ago)
+    if (lane < 9) asm volatile("cp.async.wait_group 1;" ::: "memory");     // everything but the newest group: call c is there
     __syncwarp();                                 // ... and nobody still reads the slot of call c - 2
     desc_fetch(x, slot_warp, c + 2, lane);
-    if (lane < 9) asm volatile("cp.async.commit_group;" ::: "memory");
     return warp_slot(slot_warp, c);
 }
 
