@@ -66,8 +66,9 @@ constexpr int kOffJobRec = kOffWarpDesc + kWarpRings * kDescSlots * kSlotBytes; 
 constexpr int kJobRecs = 4;
 static_assert(kOffShared + 32 <= kOffRecBar && kOffRecBar + kJobRecs * 8 <= kOffWarpDesc, "shared-memory layout");
 // finisher warps: a ring of buffers per warp that bulk copies fill with the partial sums of one row block
-constexpr int kFinSlots = 2;                  // copies in flight per finisher warp (measured on the 8B step and the
-                                              // 32-layer stack: 1: 77.8 / 562 us, 2: 79.1 / 541 us, 4: 82.7 / 580 us, 8: 88 / 651 us)
+constexpr int kFinSlots = 2;                  // copies in flight per finisher warp (measured, 8B step / 32-layer stack / a
+                                              // chain of sixteen 8B gate_up layers: 1: 71.4 / 475 / 122 us, 2: 72.2 / 482 / 107 us,
+                                              // 4: 75.6 / 494 us)
 constexpr int kFinRingBytes = 8192;           // per warp: one buffer of 32 chunks per slot
 constexpr int kOffFinBuf = (kOffJobRec + kJobRecs * 64 + 127) / 128 * 128;
 constexpr int kOffFinBar = kOffFinBuf + kFinisherWarps * kFinRingBytes;
