@@ -392,7 +392,7 @@ def _secondary(torch, elutq, name, stream, l2_bytes, hbm_peak, tensor_peak, devi
         layers.append(dict(call=c, packed=cache[key], X=X, Y=torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")))
     step_bytes = _bytes_of(calls)
     all_m1 = all(c.M == 1 for c in calls)
-    tensor = all(c.M >= 9 and c.G == 128 for c in calls)
+    tensor = all(c.M >= 9 and c.G == 128 for c in calls)           # (every call a tensor-core contraction at any N)
     # distinct blobs are shared between the calls of a step here, so rotate whole copies only while they are small
     distinct = sum(t.numel() for t in cache.values())
     out = {"workload": WORKLOAD_NAMES[name], "calls_per_step": len(calls), "algorithmic_bytes_per_step": step_bytes,

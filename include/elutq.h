@@ -65,8 +65,16 @@ typedef enum elutq_status {
                                    indices with the top bit clear and the other half is obtained by
                                    negation; same product up to fp32 rounding                              */
 
-#define ELUTQ_TENSOR_MIN_M 9      /* smallest batch that takes the tensor-core path (measured crossover: the two
-                                     paths are level at M = 8, the tensor cores win from M = 9 on)          */
+#define ELUTQ_TENSOR_MIN_M 9      /* batches of this many rows or more take the tensor-core path (G = 128, no
+                                     look-up variant flag): the batched look-up kernel needs one pass per 4 rows,
+                                     the tensor-core kernel's time does not depend on M up to 128              */
+#define ELUTQ_TENSOR_MIN_M_NARROW 5   /* ... and so do batches of 5 to 8 rows when N <= ELUTQ_TENSOR_NARROW_N: there  */
+#define ELUTQ_TENSOR_NARROW_N 8192    /* the second look-up pass already costs more than the tensor-core call (measured
+                                         on the 8B shapes at M = 8, q = 2 / 3, us: qkv 6144 x 4096 17.1 / 20.8 against
+                                         15.4 / 17.7, o 4096 x 4096 13.4 / 16.8 against 11.7 / 13.3, down 4096 x 14336
+                                         27.3 / 36.3 against 26.3 / 32.0; gate_up 28672 x 4096 43.9 / 60.6 against
+                                         48.8 / 66.5 stays on the look-up kernel).  elutq_takes_tensor_path says which
+                                         path a call takes.                                                    */
 
 #define ELUTQ_FLAG_LUT_ONLY 0x80u /* M >= 9: stay on the look-up-table kernels.  Without this flag batches of
                                      ELUTQ_TENSOR_MIN_M rows or more (G = 128) take the dequantise-and-contract path: the
@@ -250,6 +258,10 @@ int elutq_lut_gemm_host(const void* X_host, const void* packed, void* Y_host,
  *   - `packed` must be known to the library (packed or described in this process) before a capture
  *     begins: an unknown address makes the call read the header with a synchronous copy.
  */
+/* 1 when elutq_lut_gemm (and _f32, _ws, _host, _bias) runs a call of this shape on the tensor-core path, 0 when on the
+ * look-up kernels; host-only, launches nothing.  (The tensor-core path's results carry the fp16 rounding of W_hat.) */
+int elutq_takes_tensor_path(int M, int N, int K, int G, unsigned flags);
+
 int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int N, int K, void* stream);
 
 /*

@@ -54,6 +54,7 @@ _SIGNATURES = {
     "elutq_lut_gemm_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_uint, c_void_p, c_size_t, c_void_p]),
     "elutq_lut_gemm_host": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
     "elutq_lut_gemm_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]),
+    "elutq_takes_tensor_path": (c_int, [c_int, c_int, c_int, c_int, c_uint]),
     "elutq_hlq_fit": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "elutq_chain_plan_bytes": (c_int, [ctypes.POINTER(GemvCall), c_int, ctypes.POINTER(c_size_t)]),
     "elutq_chain_plan": (c_int, [ctypes.POINTER(GemvCall), c_int, c_void_p, c_size_t, c_void_p]),
@@ -185,6 +186,11 @@ def elutq_lut_gemm_ws(X, packed, Y, M: int, N: int, K: int, flags: int, workspac
 def elutq_lut_gemm_host(X_host, packed, Y_host, M: int, N: int, K: int, stream=None) -> None:
     _check(lib().elutq_lut_gemm_host(_ptr(X_host), _ptr(packed), _ptr(Y_host), M, N, K, _stream(stream)),
            "elutq_lut_gemm_host")
+
+
+def elutq_takes_tensor_path(M: int, N: int, K: int, G: int = 128, flags: int = 0) -> bool:
+    """True when elutq_lut_gemm runs this shape on the tensor-core path (host-only)."""
+    return bool(lib().elutq_takes_tensor_path(M, N, K, G, flags))
 
 
 def elutq_lut_gemm_static(X, packed, Y, M: int, N: int, K: int, stream=None) -> None:

@@ -163,6 +163,14 @@ int launch_copy_in(const void* src, void* dst, size_t bytes, cudaStream_t stream
     return (int)e;
 }
 
+// Which kernel family a batched call runs on (the crossover depends on the shape: see ELUTQ_TENSOR_MIN_M_NARROW).
+bool takes_tensor_path(int M, int N, int G, unsigned flags) {
+    const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY |
+                                  ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8;
+    if (G != 128 || (flags & lut_variants)) return false;
+    return M >= ELUTQ_TENSOR_MIN_M || (M >= ELUTQ_TENSOR_MIN_M_NARROW && N <= ELUTQ_TENSOR_NARROW_N);
+}
+
 int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, unsigned flags,
              void* workspace, size_t workspace_bytes, bool own_workspace, void* stream) {
     if (!X || !packed || !Y) return ELUTQ_ERR_INVALID_ARG;
@@ -208,10 +216,8 @@ int run_gemm(const void* X, const void* packed, void* Y, int M, int N, int K, un
     a.items_q = 0; a.items_r = 0; a.active_warps = 0; a.ranges = 0; a.rb_q = 0; a.rb_r = 0; a.cpc = 1; a.cluster_reduce = 0;
     const int sms = num_sms();
     int ce;
-    const unsigned lut_variants = ELUTQ_FLAG_PLAIN_G4 | ELUTQ_FLAG_CLUSTER_REDUCE | ELUTQ_FLAG_MIRROR | ELUTQ_FLAG_LUT_ONLY |
-                                  ELUTQ_FLAG_TABLE_F16 | ELUTQ_FLAG_TABLE_I8;
     if (M == 1) ce = launch_lut_gemv(a, m.q, m.G, sms, (cudaStream_t)stream);
-    else if (M >= ELUTQ_TENSOR_MIN_M && m.G == 128 && !(flags & lut_variants)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
+    else if (takes_tensor_path(M, N, m.G, flags)) ce = launch_hlq_mma(a, m.q, m.G, sms, (cudaStream_t)stream);
     else ce = launch_lut_gemm(a, m.q, m.G, sms, (cudaStream_t)stream);
     if (ce == (int)cudaErrorNotSupported) return ELUTQ_ERR_UNSUPPORTED;
     if (ce != 0) return cuda_fail((cudaError_t)ce);
@@ -426,6 +432,11 @@ int elutq_release_scratch(void) {
     g_parked.clear();
     if (first != cudaSuccess) return cuda_fail(first);
     return ELUTQ_OK;
+}
+
+int elutq_takes_tensor_path(int M, int N, int K, int G, unsigned flags) {
+    (void)K;
+    return M > 1 && takes_tensor_path(M, N, G, flags) ? 1 : 0;
 }
 
 int elutq_reserve(int M, int N, int K, void* stream) {

@@ -37,8 +37,9 @@ def test_batched_gemm_matches_oracle(q, G, N, K, M):
     assert_elementwise(y32, ref, A, q, K, False, False, "batched look-up kernel, fp32 out")
     y16 = gemm_f16(X, packed, N, K)                                # default path
     assert hlq.rel_fro_error(y16, ref) <= TOL_F16
-    assert_elementwise(y16, ref, A, q, K, M >= 9 and G == 128, True, "default path, fp16 out")
-    if M < 9 or G != 128:                                # below the tensor-core threshold: the same kernels
+    tensor_path = elutq.elutq_takes_tensor_path(M, N, K, G)
+    assert_elementwise(y16, ref, A, q, K, tensor_path, True, "default path, fp16 out")
+    if not tensor_path:                                  # on the look-up kernels by default: the same kernels
         assert np.array_equal(y16.view(np.uint16), y32.astype(np.float16).view(np.uint16))
 
 
@@ -47,7 +48,7 @@ def test_batched_rows_equal_single_row_calls_up_to_rounding():
     layer = workloads.hlq_layer(21, "gemm/rows", q, G, N, K)
     X = synth.activations(21, "gemm/rows/x", M, K)
     packed = pack_layer(layer)
-    yb = gemm_f32(X, packed, N, K)
+    yb = gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY)            # (a narrow layer at M = 6 would take the tensor cores by default)
     for m in range(M):
         y1 = gemm_f32(X[m:m + 1], packed, N, K)
         np.testing.assert_allclose(yb[m], y1[0], rtol=0, atol=4e-6 * np.abs(y1).max())

@@ -189,5 +189,8 @@ def test_small_batch_rows_match_oracle():
     X = synth.activations(7, "batch/x", 5, K, outliers=True)
     packed = pack_layer(layer)
     ref = hlq.matmul(X, layer.planes, layer.scales, layer.offsets, G)
-    assert hlq.rel_fro_error(gemm_f32(X, packed, N, K), ref) <= TOL_F32
+    # (five rows on a narrow layer take the tensor-core path by default: fp16 rounding of W_hat; the look-up kernels
+    #  on request are exact up to fp32 accumulation)
+    assert hlq.rel_fro_error(gemm_f32(X, packed, N, K), ref) <= (TOL_F16 if elutq.elutq_takes_tensor_path(5, N, K, G) else TOL_F32)
+    assert hlq.rel_fro_error(gemm_f32(X, packed, N, K, elutq.FLAG_LUT_ONLY), ref) <= TOL_F32
     assert hlq.rel_fro_error(gemm_f16(X, packed, N, K), ref) <= TOL_F16
