@@ -39,6 +39,67 @@ struct BCfg {
     static constexpr int SMEM_BYTES = TABLE_BYTES + (256 / G) * MB * 4 + (TQ == 2 ? 2 * MB * 4 : 0) + 64;
 };
 
+// Pieces shared by the three table builders below.  A thread owns byte-column `lane` of the half chunk (8 consecutive
+// activations) for a pair of activation rows, held as float2 (row m, row m + 1) per activation.
+
+// x[i] = (x_i of row m, x_i of row m + 1) for the 8 activations from column k0 on; rows >= M and columns >= K are zeros.
+__device__ __forceinline__ void load_row_pair(float2 (&x)[8], const __half* __restrict__ X, int M, int K, int m, int k0) {
+    float xa[8], xb[8];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        float* dst = r ? xb : xa;
+        if (m + r < M && k0 < K) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)(m + r) * K + k0);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                dst[2 * i] = f.x;
+                dst[2 * i + 1] = f.y;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = 0.f;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = make_float2(xa[i], xb[i]);
+}
+
+// The entries of the thread's 8 table rows (high nibble hi, low nibble 8*lh + t) are A[t] + Bv: A[t] = the sum of
+// x_0..x_2 selected by the bits of t (plus x_3 for the upper half of the low nibble), Bv = the sum of x_4..x_7
+// selected by the bits of hi.
+__device__ __forceinline__ void half_table_sums(float2 (&A)[8], float2& Bv, const float2 (&x)[8], int hi, int lh) {
+    A[0] = lh ? x[3] : make_float2(0.f, 0.f);
+    A[1] = fadd2(A[0], x[0]);
+    A[2] = fadd2(A[0], x[1]);
+    A[3] = fadd2(A[1], x[1]);
+    A[4] = fadd2(A[0], x[2]);
+    A[5] = fadd2(A[1], x[2]);
+    A[6] = fadd2(A[2], x[2]);
+    A[7] = fadd2(A[3], x[2]);
+    Bv = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+        if ((hi >> b) & 1) Bv = fadd2(Bv, x[4 + b]);
+}
+
+// Entry 255 (warp 31) is the column's activation sum: reduced over the W columns of a quantisation group, it gives
+// the group sums of the offset term for the two rows of the pair, gsum[group][row], row = `row` and `row` + 1 of MB.
+template <int W, int MB>
+__device__ __forceinline__ void store_group_sums(float* gsum, const float2 e255, int lane, int row) {
+    float sx = e255.x, sy = e255.y;
+#pragma unroll
+    for (int off = W / 2; off >= 1; off >>= 1) {
+        sx += __shfl_xor_sync(0xffffffffu, sx, off);
+        sy += __shfl_xor_sync(0xffffffffu, sy, off);
+    }
+    if ((lane % W) == 0) {
+        gsum[(lane / W) * MB + row] = sx;
+        gsum[(lane / W) * MB + row + 1] = sy;
+    }
+}
+
 // Tables of half chunk kc2 for rows m0 .. m0+MB-1: lane -> column c (8 activations of every row),
 // warp -> high nibble hi = warp & 15 and low-nibble half lh = warp >> 4.  Rows are paired in the
 // packed adds.  Rows >= M and columns >= K contribute zeros.
@@ -51,48 +112,13 @@ __device__ __forceinline__ void build_tables_mb(uint8_t* smem, int table_bytes, 
     const int lane = tid & 31, warp = tid >> 5;
     const int hi = warp & 15, lh = warp >> 4;
     const int k0 = kc2 * kHalfK + lane * 8;
-    float2 x[NP][8];                                    // x[p][i] = (x_i of row m0+2p, x_i of row m0+2p+1)
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-        float xa[8], xb[8];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int m = m0 + 2 * p + r;
-            float* dst = r ? xb : xa;
-            if (m < M && k0 < K) {
-                const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
-                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-                    dst[2 * i] = f.x;
-                    dst[2 * i + 1] = f.y;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) dst[i] = 0.f;
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
-    }
-    float2 e7[NP];
     uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * (4 * MB) + lane * (4 * MB);
     float2 A[NP][8], Bv[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-        A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
-        A[p][1] = fadd2(A[p][0], x[p][0]);
-        A[p][2] = fadd2(A[p][0], x[p][1]);
-        A[p][3] = fadd2(A[p][1], x[p][1]);
-        A[p][4] = fadd2(A[p][0], x[p][2]);
-        A[p][5] = fadd2(A[p][1], x[p][2]);
-        A[p][6] = fadd2(A[p][2], x[p][2]);
-        A[p][7] = fadd2(A[p][3], x[p][2]);
-        Bv[p] = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int b = 0; b < 4; ++b)
-            if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+        float2 x[8];
+        load_row_pair(x, X, M, K, m0 + 2 * p, k0);
+        half_table_sums(A[p], Bv[p], x, hi, lh);
     }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -102,24 +128,9 @@ __device__ __forceinline__ void build_tables_mb(uint8_t* smem, int table_bytes, 
         uint8_t* dst = rowp + (size_t)t * 32 * (4 * MB);
         if (MB == 2) *reinterpret_cast<float2*>(dst) = e[0];
         else *reinterpret_cast<float4*>(dst) = make_float4(e[0].x, e[0].y, e[NP - 1].x, e[NP - 1].y);
-        if (t == 7) {
+        if (t == 7 && warp == 31) {
 #pragma unroll
-            for (int p = 0; p < NP; ++p) e7[p] = e[p];
-        }
-    }
-    if (warp == 31) {   // entry 255: the column's activation sums; reduce over the W columns of a group
-#pragma unroll
-        for (int p = 0; p < NP; ++p) {
-            float sx = e7[p].x, sy = e7[p].y;
-#pragma unroll
-            for (int off = W / 2; off >= 1; off >>= 1) {
-                sx += __shfl_xor_sync(0xffffffffu, sx, off);
-                sy += __shfl_xor_sync(0xffffffffu, sy, off);
-            }
-            if ((lane % W) == 0) {
-                gsum[(lane / W) * MB + 2 * p] = sx;
-                gsum[(lane / W) * MB + 2 * p + 1] = sy;
-            }
+            for (int p = 0; p < NP; ++p) store_group_sums<W, MB>(gsum, e[p], lane, 2 * p);
         }
     }
 }
@@ -139,46 +150,12 @@ __device__ __forceinline__ void build_tables_half(uint8_t* smem, int table_bytes
     uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * EB + lane * EB;
 #pragma unroll 1
     for (int quad = 0; quad < MB / 4; ++quad) {
-        float2 x[2][8];                                 // x[p][i] = (x_i of row m0+4quad+2p, x_i of the next row)
+        float2 A[2][8], Bv[2];
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-            float xa[8], xb[8];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int m = m0 + 4 * quad + 2 * p + r;
-                float* dst = r ? xb : xa;
-                if (m < M && k0 < K) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
-                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-                        dst[2 * i] = f.x;
-                        dst[2 * i + 1] = f.y;
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) dst[i] = 0.f;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
-        }
-        float2 A[2][8], Bv[2], e7[2];
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
-            A[p][1] = fadd2(A[p][0], x[p][0]);
-            A[p][2] = fadd2(A[p][0], x[p][1]);
-            A[p][3] = fadd2(A[p][1], x[p][1]);
-            A[p][4] = fadd2(A[p][0], x[p][2]);
-            A[p][5] = fadd2(A[p][1], x[p][2]);
-            A[p][6] = fadd2(A[p][2], x[p][2]);
-            A[p][7] = fadd2(A[p][3], x[p][2]);
-            Bv[p] = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-                if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+            float2 x[8];
+            load_row_pair(x, X, M, K, m0 + 4 * quad + 2 * p, k0);
+            half_table_sums(A[p], Bv[p], x, hi, lh);
         }
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
@@ -186,21 +163,9 @@ __device__ __forceinline__ void build_tables_half(uint8_t* smem, int table_bytes
             const __half2 ha = __floats2half2_rn(ea.x, ea.y), hb = __floats2half2_rn(eb.x, eb.y);
             *reinterpret_cast<uint2*>(rowp + (size_t)t * 32 * EB + quad * 8) =
                 make_uint2(*reinterpret_cast<const uint32_t*>(&ha), *reinterpret_cast<const uint32_t*>(&hb));
-            if (t == 7) { e7[0] = ea; e7[1] = eb; }
-        }
-        if (warp == 31) {   // entry 255: the column's activation sums; reduce over the W columns of a group
-#pragma unroll
-            for (int p = 0; p < 2; ++p) {
-                float sx = e7[p].x, sy = e7[p].y;
-#pragma unroll
-                for (int off = W / 2; off >= 1; off >>= 1) {
-                    sx += __shfl_xor_sync(0xffffffffu, sx, off);
-                    sy += __shfl_xor_sync(0xffffffffu, sy, off);
-                }
-                if ((lane % W) == 0) {
-                    gsum[(lane / W) * MB + 4 * quad + 2 * p] = sx;
-                    gsum[(lane / W) * MB + 4 * quad + 2 * p + 1] = sy;
-                }
+            if (t == 7 && warp == 31) {
+                store_group_sums<W, MB>(gsum, ea, lane, 4 * quad);
+                store_group_sums<W, MB>(gsum, eb, lane, 4 * quad + 2);
             }
         }
     }
@@ -220,38 +185,15 @@ __device__ __forceinline__ void build_tables_i8(uint8_t* smem, int table_bytes, 
     uint8_t* rowp = smem + (size_t)(hi * 16 + lh * 8) * 32 * MB + lane * MB;
 #pragma unroll 1
     for (int quad = 0; quad < 2; ++quad) {
-        float2 x[2][8];
+        float2 A[2][8], Bv[2], inv[2];
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-            float xa[8], xb[8];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int m = m0 + 4 * quad + 2 * p + r;
-                float* dst = r ? xb : xa;
-                if (m < M && k0 < K) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(X + (size_t)m * K + k0);
-                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-                        dst[2 * i] = f.x;
-                        dst[2 * i + 1] = f.y;
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) dst[i] = 0.f;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[p][i] = make_float2(xa[i], xb[i]);
-        }
-        float2 A[2][8], Bv[2], e7[2], inv[2];
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
+            float2 x[8];
+            load_row_pair(x, X, M, K, m0 + 4 * quad + 2 * p, k0);
             // largest |entry| this column can produce, then the group's maximum over its 16 columns
             float ax = 0.f, ay = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { ax += fabsf(x[p][i].x); ay += fabsf(x[p][i].y); }
+            for (int i = 0; i < 8; ++i) { ax += fabsf(x[i].x); ay += fabsf(x[i].y); }
 #pragma unroll
             for (int off = W / 2; off >= 1; off >>= 1) {
                 ax = fmaxf(ax, __shfl_xor_sync(0xffffffffu, ax, off));
@@ -262,18 +204,7 @@ __device__ __forceinline__ void build_tables_i8(uint8_t* smem, int table_bytes, 
                 rscale[(lane / W) * MB + 4 * quad + 2 * p] = ax / 127.f;
                 rscale[(lane / W) * MB + 4 * quad + 2 * p + 1] = ay / 127.f;
             }
-            A[p][0] = lh ? x[p][3] : make_float2(0.f, 0.f);
-            A[p][1] = fadd2(A[p][0], x[p][0]);
-            A[p][2] = fadd2(A[p][0], x[p][1]);
-            A[p][3] = fadd2(A[p][1], x[p][1]);
-            A[p][4] = fadd2(A[p][0], x[p][2]);
-            A[p][5] = fadd2(A[p][1], x[p][2]);
-            A[p][6] = fadd2(A[p][2], x[p][2]);
-            A[p][7] = fadd2(A[p][3], x[p][2]);
-            Bv[p] = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-                if ((hi >> b) & 1) Bv[p] = fadd2(Bv[p], x[p][4 + b]);
+            half_table_sums(A[p], Bv[p], x, hi, lh);
         }
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
@@ -281,21 +212,9 @@ __device__ __forceinline__ void build_tables_i8(uint8_t* smem, int table_bytes, 
             const uint32_t c0 = (uint32_t)(__float2int_rn(ea.x * inv[0].x) + 128), c1 = (uint32_t)(__float2int_rn(ea.y * inv[0].y) + 128);
             const uint32_t c2 = (uint32_t)(__float2int_rn(eb.x * inv[1].x) + 128), c3 = (uint32_t)(__float2int_rn(eb.y * inv[1].y) + 128);
             *reinterpret_cast<uint32_t*>(rowp + (size_t)t * 32 * MB + quad * 4) = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
-            if (t == 7) { e7[0] = ea; e7[1] = eb; }
-        }
-        if (warp == 31) {   // entry 255: the column's activation sums; reduce over the 16 columns of a group
-#pragma unroll
-            for (int p = 0; p < 2; ++p) {
-                float sx = e7[p].x, sy = e7[p].y;
-#pragma unroll
-                for (int off = W / 2; off >= 1; off >>= 1) {
-                    sx += __shfl_xor_sync(0xffffffffu, sx, off);
-                    sy += __shfl_xor_sync(0xffffffffu, sy, off);
-                }
-                if ((lane % W) == 0) {
-                    gsum[(lane / W) * MB + 4 * quad + 2 * p] = sx;
-                    gsum[(lane / W) * MB + 4 * quad + 2 * p + 1] = sy;
-                }
+            if (t == 7 && warp == 31) {
+                store_group_sums<W, MB>(gsum, ea, lane, 4 * quad);
+                store_group_sums<W, MB>(gsum, eb, lane, 4 * quad + 2);
             }
         }
     }
