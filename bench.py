@@ -9,7 +9,7 @@ printed by rank 0:
   value       achieved GB/s = algorithmic bytes of the step (bit-planes + fp16 scales + fp16 offsets +
               X + Y, summed over the calls) / device time, inputs resident in HBM.  M = 1 workloads run
               the step through the chained decode entry (elutq_chain_run: the list of calls in one
-              persistent launch per bit-width); the same step as separate elutq_lut_gemm calls replayed
+              persistent launch); the same step as separate elutq_lut_gemm calls replayed
               from a CUDA graph is timed beside it (`secondary`).  The working set of a step exceeds
               the L2 capacity
   e2e         the same metric through elutq_lut_gemm_host: X copied from pinned host memory and Y copied

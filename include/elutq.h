@@ -269,8 +269,9 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  *
  * At M = 1 every linear of a decode step is one bit-serial LUT GEMV; launched one by one, each pays its own
  * kernel start, K-split reduction and kernel end, during which HBM idles.  A chain runs a fixed list of
- * such calls - typically all linears of a decode step, in model order - in ONE persistent launch (one per run
- * of consecutive calls with equal (q, G): a model has one such pair, a mixed list is cut at the changes):
+ * such calls - typically all linears of a decode step, in model order - in ONE persistent launch (calls of
+ * G = 128 may mix bit-widths freely; for other group sizes a launch takes a run of consecutive calls with equal
+ * (q, G), and a list is cut where the group size changes):
  * Y_c[N_c] = X_c[K_c] * W_hat_c^T for c = 0 .. n_calls-1, each result identical in value to elutq_lut_gemm
  * up to the order of the fp32 K-chunk sum (chunks are always added in ascending order, so a chain is
  * bit-reproducible from launch to launch).
@@ -290,7 +291,7 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  *                           Pointers and shapes are frozen in the plan; the buffers they name may change
  *                           content between runs.  M is 1; flags per call: ELUTQ_FLAG_OUT_F32,
  *                           ELUTQ_FLAG_ACCUMULATE (others: ELUTQ_ERR_UNSUPPORTED).
- *   elutq_chain_run         one launch on `stream` per run of equal (q, G) (one CTA per SM; the first launch is
+ *   elutq_chain_run         one launch on `stream` per run, normally one in all (one CTA per SM; the first launch is
  *                           cooperative: the device must be able to hold its CTAs all at once, else
  *                           ELUTQ_ERR_CUDA and nothing runs).  Allocates nothing.  Runs of one plan must not
  *                           overlap on the GPU.  Every CTA first compares the header of each blob of its launch
@@ -334,7 +335,7 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* str
 int elutq_chain_run_host(void* plan, int n_calls, void* x_dev, const void* x_host, size_t x_bytes, const void* y_dev,
                          void* y_host, size_t y_bytes, void* stream);
 int elutq_chain_status(const void* plan, void* stream, int* status);
-/* The library keeps a small host-side note per planned buffer (which runs of equal (q, G) to launch);
+/* The library keeps a small host-side note per planned buffer (which runs of calls to launch);
  * elutq_chain_run returns ELUTQ_ERR_SHAPE for a buffer that this process has not planned.  Call this before
  * freeing a plan buffer. */
 int elutq_chain_forget(const void* plan);

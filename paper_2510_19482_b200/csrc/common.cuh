@@ -102,6 +102,18 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const void* p) {
     asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1+%2];" : "=r"(v) : "l"(p), "n"(IMM));
     return v;
 }
+// The same loads under a run-time condition (on == 0: no access, the registers keep their values).
+template <int IMM>
+__device__ __forceinline__ void ldg_stream_v4_if(uint4& v, const void* p, uint32_t on) {
+    asm volatile("{\n\t.reg .pred pq;\n\tsetp.ne.u32 pq, %6, 0;\n\t"
+                 "@pq ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4+%5];\n\t}"
+                 : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "l"(p), "n"(IMM), "r"(on));
+}
+template <int IMM>
+__device__ __forceinline__ void ldg_stream_u32_if(uint32_t& v, const void* p, uint32_t on) {
+    asm volatile("{\n\t.reg .pred pq;\n\tsetp.ne.u32 pq, %3, 0;\n\t"
+                 "@pq ld.global.nc.L1::no_allocate.u32 %0, [%1+%2];\n\t}" : "+r"(v) : "l"(p), "n"(IMM), "r"(on));
+}
 // Compile-time loop: f(IntC<I>) for I in [0, N); IntC<I> converts to a constant int.
 template <int V>
 struct IntC {

@@ -3,9 +3,9 @@
 // A decode step is a fixed sequence of linears on one stream.  Launched one by one, every call pays its own
 // chain of cross-SM hand-overs (kernel start, activation load, table build, K-split reduction, kernel end), during
 // which HBM idles; for the 8B layer shapes that chain is several times longer than the time the call's bytes need.
-// Here one grid (one 1024-thread CTA per SM, all resident) walks a run of consecutive calls that share (q, G) - a
-// model has one such pair, so normally the whole list is one launch; a list that mixes them is cut into one
-// launch per run.  Inside a CTA the warps are specialised (Appendix B's two phases run side by side):
+// Here one grid (one 1024-thread CTA per SM, all resident) walks a run of consecutive calls: calls of G = 128 with
+// any mix of bit-widths, or calls that share (q, G) for the other group sizes - normally the whole list is one launch;
+// a list that mixes group sizes is cut into one launch per run.  Inside a CTA the warps are specialised (Appendix B's two phases run side by side):
 //
 //   * 4 builder warps, as two teams of two (team t: the table jobs of parity t, always in table buffer t), load the
 //     activations of the CTA's next K chunk and fill the table buffers (fused 8-bit tables, 64 KiB each); before a
@@ -74,7 +74,7 @@ constexpr int kOffFinBuf = (kOffJobRec + kJobRecs * 64 + 127) / 128 * 128;
 constexpr int kOffFinBar = kOffFinBuf + kFinisherWarps * kFinRingBytes;
 constexpr int kChainSmem = kOffFinBar + kFinisherWarps * kFinSlots * 8;
 constexpr unsigned kCallTestNoSignal = 0x40000000u;   // test only: the call never reports completion
-constexpr int kMaxRuns = 64;                  // launches per chain (runs of equal (q, G))
+constexpr int kMaxRuns = 64;                  // launches per chain
 
 struct ChainCtl {                             // first 256 bytes of a plan
     unsigned magic, n_calls, status, epoch;
@@ -162,7 +162,8 @@ struct JobRec {                               // four 16-byte quarters, each rea
     int N;
     unsigned flags;
     unsigned tag;
-    int last;                                 // bit 0: the call's last job on this CTA; bit 1: the call's report is a release
+    int last;                                 // bit 0: the call's last job on this CTA; bit 1: the call's report is a release;
+                                              // bits 8 and up: the call's bit-width q
     int stop;                                 // 1: no more jobs in this launch
     int out_stride;                           // 64-bit words from one row block's partial sums to the next (16 n_kc)
 };
@@ -474,14 +475,27 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 // At its last item of the job the warp looks for the record of the next job (the builders publish it before they
 // build that job's tables, normally a whole job ahead): if it is there and gives the warp an item, that item's loads
 // ride along with the last item and `buf` holds it on exit (returns true).
-template <int Q, int G, int B>
-__device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
+// Q = 0: the bit-width is the job's (q, from its record; G = 128), and the next job's may differ.
+template <int Q, int G>
+struct ItemOf { using type = Item<Q, G>; };
+template <int G>
+struct ItemOf<0, G> { using type = ItemRt; };
+
+template <int Q, int G>
+__device__ __forceinline__ int chain_tile_bytes(int q) { return Q ? Cfg<Q ? Q : 1, G>::TILE_BYTES : tile_bytes_g128(q); }
+
+// QC: the job's bit-width as a compile-time value (= Q for a kernel of one bit-width; for Q = 0, the run-time-q kernel,
+// the caller switches on the job's q, and only an item whose successor belongs to a job of another q takes a form
+// with conditional loads).
+template <int Q, int QC, int G, int B>
+__device__ __forceinline__ bool chain_items(typename ItemOf<Q, G>::type& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
                                             unsigned long long* out, void* Y, const int N, const unsigned flags,
                                             const unsigned tag, const int out_stride, const uint8_t* vp, const unsigned job,
-                                            const size_t warp_off, const int lw, const int lane) {
-    using C = Cfg<Q, G>;
-    const uint8_t* const tab = chain_smem + B * kTableBytes;
-    const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + B * 64);
+                                            const size_t warp_off, const int lw, const int lane, const int b_rt) {
+    using C = Cfg<QC, G>;
+    const int bb = B < 0 ? b_rt : B;
+    const uint8_t* const tab = chain_smem + bb * kTableBytes;
+    const float* gsum = reinterpret_cast<const float*>(chain_smem + kOffGsum + bb * 64);
     const int h = lane >> 4, l = lane & 15;
     float S[C::GL];
     load_group_sums<G>(S, gsum, h, l, true);
@@ -490,17 +504,26 @@ __device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&co
     for (int rb = rb0 + lw; rb < rb1; rb += kLookupWarps) {
         const bool in_job = rb + kLookupWarps < rb1;
         const uint8_t* nvp = vp + kLookupWarps * C::TILE_BYTES;
+        int nq = QC;
         if (!in_job && __all_sync(0xffffffffu, mbar_test(bar_rec(job + 1), ((job + 1) >> 2) & 1u))) {
             const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
             if ((int)n0.z + lw < (int)n0.w) {
-                nvp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + warp_off;
-                carried = true;
+                size_t noff = warp_off;
+                if constexpr (Q == 0) nq = job_rec(job + 1)->last >> 8;
+                if (nq == QC) {               // (a job of another q: its first item is requested when the job begins)
+                    nvp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + noff;
+                    carried = true;
+                }
             }
         }
-        const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
         float y;
-        if (in_job || carried) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
-        else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
+        if constexpr (Q == 0) {
+            y = item_sum_rt<QC>(buf, tab, colp, S, nvp, (in_job || carried) ? 1u : 0u, lane);
+        } else {
+            const uint8_t* npp = nvp + (C::PLANE_BYTES - lane * 12);
+            if (in_job || carried) y = item_sum<Q, G, kModeFused, true>(buf, tab, colp, S, nvp, npp, true, true);
+            else y = item_sum<Q, G, kModeFused, false>(buf, tab, colp, S, nvp, npp, true, true);
+        }
         if (h == 0) {
             if (out == nullptr) {
                 if (rb * kTileRows + l < N) chain_store(Y, flags, (size_t)(rb * kTileRows + l), y);
@@ -511,6 +534,16 @@ __device__ __forceinline__ bool chain_items(Item<Q, G>& buf, const uint32_t (&co
         vp = nvp;
     }
     return carried;
+}
+
+// the job's items, tables in buffer b
+template <int Q, int QC, int G>
+__device__ __forceinline__ bool chain_items_b(int b, typename ItemOf<Q, G>::type& buf, const uint32_t (&colp)[4], const int rb0,
+                                              const int rb1, unsigned long long* out, void* Y, const int N, const unsigned flags,
+                                              const unsigned tag, const int out_stride, const uint8_t* vp, const unsigned job,
+                                              const size_t warp_off, const int lw, const int lane) {
+    if (b == 0) return chain_items<Q, QC, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 0);
+    return chain_items<Q, QC, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 1);
 }
 
 // What the roles of a launch share.
@@ -545,20 +578,22 @@ __device__ __forceinline__ const ChainSlot* desc_next(const ChainCtx& x, int slo
     return warp_slot(slot_warp, c);
 }
 
-// Look-up role of one warp: it follows the job records the builders publish.  (A launch covers calls of one (q, G):
-// a variant that switched between per-q instances of this function inside one kernel was measured three times slower,
-// whether the instances were inlined or called.)
+// Look-up role of one warp: it follows the job records the builders publish.  Q = 0 is the kernel for lists that mix
+// bit-widths (G = 128): one register buffer sized for q = 4, and per job a switch to the straight-line code for the
+// job's q.  What made that form as fast as a kernel of one q (earlier forms were 1.2 to 3 times slower): the buffer
+// is shared by the per-q bodies instead of one buffer type per q (those spilled 0.3-1.5 KB per thread); a body per q
+// and table buffer but none per "has a next item" (a predicate on the refill loads instead); the table buffer a
+// compile-time constant (a run-time base costs an add per look-up); the unused part of the buffer given a value
+// after every job.
 template <int Q, int G>
 __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
-    using C = Cfg<Q, G>;
     const int lane = threadIdx.x & 31, lw = threadIdx.x >> 5;
     const int h = lane >> 4, l = lane & 15;
     ChainShared* sh = chain_shared();
     uint32_t colp[4];
     make_colp<G>(colp, h, l);
-    Item<Q, G> buf;
+    typename ItemOf<Q, G>::type buf;
     bool carried = false;                     // buf already holds this warp's first item of the job
-    const size_t warp_off = (size_t)lw * C::TILE_BYTES + lane * 16;
     for (unsigned job = 0;; ++job) {
         const int b = job & 1;
         // The job's record comes before its tables: the warp requests its first item of the job (unless the item came
@@ -577,13 +612,40 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
         const int N = (int)q2.z;
         const unsigned flags = q2.w, tag = q3.x;
         const int out_stride = (int)q3.w;
-        const bool items = rb0 + lw < rb1;
-        const uint8_t* vp = tile0 + warp_off;
-        if (items && !carried) load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
-        mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
-        if (sh->abort) break;
-        if (b == 0) carried = chain_items<Q, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
-        else carried = chain_items<Q, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
+        // (for Q = 0 everything from here on exists once per bit-width, behind a switch on the job's q)
+        auto run_job = [&](auto qc) -> bool {
+            constexpr int QC = decltype(qc)::value;
+            using C = Cfg<QC, G>;
+            const size_t warp_off = (size_t)lw * C::TILE_BYTES + lane * 16;
+            const uint8_t* vp = tile0 + warp_off;
+            if (rb0 + lw < rb1 && !carried) {
+                if constexpr (Q == 0) load_item_rt<QC>(buf, vp, lane);
+                else load_item<Q, G>(buf, vp, vp + (C::PLANE_BYTES - lane * 12), true);
+            }
+            mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
+            if (sh->abort) return false;
+            carried = chain_items_b<Q, QC, G>(b, buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
+            if constexpr (Q == 0) {
+                // the part of the buffer that items of this q do not use: given a value here, it is known not to carry one
+                // through the job, which leaves its registers to the look-ups (without this the bodies for q < 4 ran 8 %
+                // slower than a kernel of that q alone)
+                static_for<QC, 4>([&](auto j) { buf.v[0][j] = make_uint4(0u, 0u, 0u, 0u); buf.v[1][j] = make_uint4(0u, 0u, 0u, 0u); });
+                static_for<QC + 1, 5>([&](auto i) { buf.p[i] = 0u; });
+            }
+            return true;
+        };
+        bool went;
+        if constexpr (Q == 0) {
+            switch (q3.y >> 8) {
+                case 1: went = run_job(IntC<1>{}); break;
+                case 2: went = run_job(IntC<2>{}); break;
+                case 3: went = run_job(IntC<3>{}); break;
+                default: went = run_job(IntC<4>{}); break;
+            }
+        } else {
+            went = run_job(IntC<Q>{});
+        }
+        if (!went) break;
         const bool report = out == nullptr && (q3.y & 1u) != 0u && !(flags & kCallTestNoSignal);
         __syncwarp();
         if (lane == 0) {
@@ -683,10 +745,10 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         // the first tables meanwhile.
         {
             int hdr_bad = 0;
-            if (hdr_mine && (hdr_q != Q || hdr_g != G || !blob_header_ok(hdr0, hdr1, Q, G, hdr_n, hdr_k))) hdr_bad = 1;
+            if (hdr_mine && ((Q ? hdr_q != Q : (hdr_q < 1 || hdr_q > 4)) || hdr_g != G || !blob_header_ok(hdr0, hdr1, hdr_q, G, hdr_n, hdr_k))) hdr_bad = 1;
             for (int c = c_begin + kHdrThreads + tid; c < c_end; c += kLookupWarps * 32) {      // launches of more calls
                 const ChainCall* d = calls + c;
-                if (d->q != Q || d->G != G || !blob_header_matches(d->tiles, Q, G, d->N, d->K, nullptr)) hdr_bad = 1;
+                if ((Q ? d->q != Q : (d->q < 1 || d->q > 4)) || d->G != G || !blob_header_matches(d->tiles, d->q, G, d->N, d->K, nullptr)) hdr_bad = 1;
             }
             if (hdr_bad) sh->headers_bad = 1;
             bar_lookups();
@@ -738,7 +800,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
                         // read four jobs ago)
                         JobRec* r = job_rec(j);
                         const int kc = p.kc0 + seg;
-                        r->tile0 = d->tiles + ((size_t)kc * d->n_rb + p.rb0) * Cfg<Q, G>::TILE_BYTES;
+                        r->tile0 = d->tiles + ((size_t)kc * d->n_rb + p.rb0) * chain_tile_bytes<Q, G>(d->q);
                         r->out = d->n_kc > 1 ? d->slots + (size_t)kc * kTileRows : nullptr;
                         r->out_stride = d->n_kc * kTileRows;
                         r->Y = d->Y;
@@ -746,7 +808,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
                         r->rb0 = p.rb0; r->rb1 = p.rb1; r->N = d->N;
                         r->flags = d->flags;
                         r->tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
-                        r->last = (seg + 1 == nseg ? 1 : 0) | (d->release ? 2 : 0);
+                        r->last = (seg + 1 == nseg ? 1 : 0) | (d->release ? 2 : 0) | (d->q << 8);
                         r->stop = 0;
                         __threadfence_block();
                         mbar_arrive(bar_rec(j));
@@ -899,7 +961,7 @@ cudaError_t launch_run_q(int G, ChainCtl* ctl, const ChainCall* calls, const int
     }
 }
 
-// Host-side copy of what elutq_chain_run needs of a plan (the runs of equal (q, G)), keyed by the plan's device
+// Host-side copy of what elutq_chain_run needs of a plan (its runs: consecutive calls of G = 128, or of equal (q, G)), keyed by the plan's device
 // address; written by elutq_chain_plan.
 struct PlanRuns {
     int n_calls = 0;
@@ -1004,7 +1066,9 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
         d.guard_call = i >= kChainRegions ? i - kChainRegions : -1;
         d.guard_target = d.guard_call >= 0 ? dc[d.guard_call].done_target : 0u;
         d.done_target = (unsigned)(g.n_kc > 1 ? d.n_ctas : d.n_ctas * kLookupWarps);
-        if (runs.n_runs == 0 || runs.q[runs.n_runs - 1] != q || runs.G[runs.n_runs - 1] != G) {
+        if (runs.n_runs > 0 && G == 128 && runs.G[runs.n_runs - 1] == 128 && runs.q[runs.n_runs - 1] != q) {
+            runs.q[runs.n_runs - 1] = 0;      // consecutive calls of G = 128 and different q: one launch of the run-time-q kernel
+        } else if (runs.n_runs == 0 || runs.q[runs.n_runs - 1] != q || runs.G[runs.n_runs - 1] != G) {
             if (runs.n_runs == kMaxRuns) return ELUTQ_ERR_UNSUPPORTED;
             runs.begin[runs.n_runs] = i;
             runs.q[runs.n_runs] = q;
@@ -1045,6 +1109,7 @@ int elutq_chain_run_opts(void* plan, int n_calls, unsigned wait_limit, void* str
         const int last = r + 1 == runs.n_runs;
         cudaError_t e;
         switch (runs.q[r]) {
+            case 0: e = launch_run<0, 128>(ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
             case 1: e = launch_run_q<1>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
             case 2: e = launch_run_q<2>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;
             case 3: e = launch_run_q<3>(runs.G[r], ctl, calls, parts, done, n_calls, runs.begin[r], runs.begin[r + 1], r == 0, last, wait_limit, sms, (cudaStream_t)stream); break;

@@ -275,6 +275,80 @@ __device__ __forceinline__ float item_sum(Item<Q, G>& buf, const uint8_t* smem, 
     return y;
 }
 
+// ---- Items of different bit-widths through one register buffer (G = 128, fused tables), for a kernel that serves a
+// list of calls of mixed q: the buffer is sized for q = 4, and one straight-line body per q works on it (the caller
+// switches on the job's q).  A tile holds, per lane, 2 q plane vectors (vector (u, j) = plane j of the lane's half u,
+// 512 bytes apart, half 1 after the q vectors of half 0) and q + 1 parameter words (fp16 pairs: s_0 .. s_{q-1}, z of
+// half 0, then the same of half 1).  The look-ups and the order of the additions are those of item_sum, so the results
+// are bit-identical.  Whether a next item exists is a run-time predicate on the refill loads (no second body).
+struct ItemRt {
+    uint4 v[2][4];
+    uint32_t p[5];
+};
+
+constexpr __host__ __device__ int tile_bytes_g128(int q) { return 1024 * q + 128 * (q + 1); }
+
+// vp = tile + lane * 16
+template <int QC>
+__device__ __forceinline__ void load_item_rt(ItemRt& it, const uint8_t* vp, int lane) {
+    static_for<0, 2 * QC>([&](auto i) { it.v[i / QC][i % QC] = ldg_stream_v4<i * 512>(vp); });
+    const uint8_t* pp = vp + (QC * 1024 - lane * 12);
+    static_for<0, QC + 1>([&](auto i) { it.p[i] = ldg_stream_u32<i * 128>(pp); });
+}
+
+// sum of the 16 table entries one plane vector selects (the lane's 16 byte-columns of half U)
+template <int U>
+__device__ __forceinline__ float plane_lookups(const uint4& vec, const uint8_t* tab, const uint32_t (&colp)[4]) {
+    const uint32_t wd[4] = {vec.x, vec.y, vec.z, vec.w};
+    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int ii = 0; ii < 16; ii += 2) {
+        float e[2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int i = ii + t;
+            const uint32_t off = prmt(wd[i >> 2], colp[i >> 2], 0xCC04 + 0x11 * (i & 3));   // (weight byte << 8) | lane column
+            e[t] = *reinterpret_cast<const float*>(tab + off + U * 128);
+        }
+        acc = fadd2(acc, make_float2(e[0], e[1]));
+    }
+    return acc.x + acc.y;
+}
+
+// One item of bit-width QC; where `next` is non-zero the registers are refilled, as they are consumed, with the item
+// at nvp (= its tile + lane * 16), which has the same bit-width.
+template <int QC>
+__device__ __forceinline__ float item_sum_rt(ItemRt& buf, const uint8_t* tab, const uint32_t (&colp)[4], const float (&S)[2],
+                                             const uint8_t* nvp, const uint32_t next, const int lane) {
+    // the scales of half 1 start at fp16 number QC + 1: bring them (and the two offsets) to fixed positions
+    uint32_t s0[2] = {buf.p[0], buf.p[1]}, s1[2] = {0u, 0u}, zz;
+    if constexpr (QC == 1) {
+        s1[0] = buf.p[1]; zz = prmt(buf.p[0], buf.p[1], 0x7632);
+    } else if constexpr (QC == 2) {
+        s1[0] = prmt(buf.p[1], buf.p[2], 0x5432); zz = prmt(buf.p[1], buf.p[2], 0x7610);
+    } else if constexpr (QC == 3) {
+        s1[0] = buf.p[2]; s1[1] = buf.p[3]; zz = prmt(buf.p[1], buf.p[3], 0x7632);
+    } else {
+        s1[0] = prmt(buf.p[2], buf.p[3], 0x5432); s1[1] = prmt(buf.p[3], buf.p[4], 0x5432);
+        zz = prmt(buf.p[2], buf.p[4], 0x7610);
+    }
+    const uint8_t* npp = nvp + (QC * 1024 - lane * 12);
+    static_for<0, QC + 1>([&](auto i) { ldg_stream_u32_if<i * 128>(buf.p[i], npp, next); });
+    float y = 0.f;
+    static_for<0, 2 * QC>([&](auto uj) {
+        constexpr int u = uj / QC, j = uj % QC;
+        const __half2 h2 = *reinterpret_cast<const __half2*>(u ? &s1[j >> 1] : &s0[j >> 1]);
+        const float sc = (j & 1) ? __high2float(h2) : __low2float(h2);
+        y = fmaf(sc, plane_lookups<u>(buf.v[u][j], tab, colp), y);
+        ldg_stream_v4_if<uj * 512>(buf.v[u][j], nvp, next);       // the vector is dead now: the next item's takes its place
+    });
+    const __half2 z2 = *reinterpret_cast<const __half2*>(&zz);
+    y = fmaf(__low2float(z2), S[0], y);
+    y = fmaf(__high2float(z2), S[1], y);
+    y += __shfl_xor_sync(0xffffffffu, y, 16);
+    return y;
+}
+
 // Aligned partition of one M = 1 call over the SMs: groups of `cpc` consecutive K chunks x R row ranges, one
 // CTA each.  Returns false when the flat cut of the item list is predicted to finish sooner.
 bool plan_gemv_partition(int n_rb, int n_kc, int num_sms, bool allow_flat, int* cpc, int* ranges);
