@@ -164,7 +164,8 @@ struct JobRec {                               // four 16-byte quarters, each rea
     unsigned tag;
     int last;                                 // bit 0: the call's last job on this CTA; bit 1: the call's report is a release;
                                               // bits 8 and up: the call's bit-width q
-    int stop;                                 // 1: no more jobs in this launch
+    int stop;                                 // bit 0: no more jobs in this launch; bits 8 and up: the look-up warp that
+                                              // takes the job's first item
     int out_stride;                           // 64-bit words from one row block's partial sums to the next (16 n_kc)
 };
 static_assert(sizeof(JobRec) == 64, "job record size");
@@ -475,6 +476,15 @@ __device__ __forceinline__ void build_tables_bw(uint8_t* tab, float* gsum, const
 // At its last item of the job the warp looks for the record of the next job (the builders publish it before they
 // build that job's tables, normally a whole job ahead): if it is there and gives the warp an item, that item's loads
 // ride along with the last item and `buf` holds it on exit (returns true).
+// Items are dealt to the look-up warps round robin ACROSS jobs: a job's first item goes to the warp after the one
+// that took the last item of the job before (`first`, from the job's record), so that short jobs (fewer items than
+// warps: the small layers) alternate between warps, and the latency of a warp's item runs beside the next job's
+// instead of in front of it.  The warp's place in a job whose first item goes to warp `first`:
+__device__ __forceinline__ int item_slot(int warp, int first) {
+    const int s = warp - first;
+    return s < 0 ? s + kLookupWarps : s;
+}
+
 // Q = 0: the bit-width is the job's (q, from its record; G = 128), and the next job's may differ.
 template <int Q, int G>
 struct ItemOf { using type = Item<Q, G>; };
@@ -491,7 +501,7 @@ template <int Q, int QC, int G, int B>
 __device__ __forceinline__ bool chain_items(typename ItemOf<Q, G>::type& buf, const uint32_t (&colp)[4], const int rb0, const int rb1,
                                             unsigned long long* out, void* Y, const int N, const unsigned flags,
                                             const unsigned tag, const int out_stride, const uint8_t* vp, const unsigned job,
-                                            const size_t warp_off, const int lw, const int lane, const int b_rt) {
+                                            const size_t warp_off, const int lw, const int lane, const int b_rt, const int wp) {
     using C = Cfg<QC, G>;
     const int bb = B < 0 ? b_rt : B;
     const uint8_t* const tab = chain_smem + bb * kTableBytes;
@@ -507,8 +517,9 @@ __device__ __forceinline__ bool chain_items(typename ItemOf<Q, G>::type& buf, co
         int nq = QC;
         if (!in_job && __all_sync(0xffffffffu, mbar_test(bar_rec(job + 1), ((job + 1) >> 2) & 1u))) {
             const uint4 n0 = *reinterpret_cast<const uint4*>(job_rec(job + 1));
-            if ((int)n0.z + lw < (int)n0.w) {
-                size_t noff = warp_off;
+            const int nlw = item_slot(wp, job_rec(job + 1)->stop >> 8);      // the warp's place in the next job
+            if ((int)n0.z + nlw < (int)n0.w) {
+                const size_t noff = (size_t)nlw * C::TILE_BYTES + lane * 16;
                 if constexpr (Q == 0) nq = job_rec(job + 1)->last >> 8;
                 if (nq == QC) {               // (a job of another q: its first item is requested when the job begins)
                     nvp = reinterpret_cast<const uint8_t*>(((unsigned long long)n0.y << 32) | n0.x) + noff;
@@ -541,9 +552,9 @@ template <int Q, int QC, int G>
 __device__ __forceinline__ bool chain_items_b(int b, typename ItemOf<Q, G>::type& buf, const uint32_t (&colp)[4], const int rb0,
                                               const int rb1, unsigned long long* out, void* Y, const int N, const unsigned flags,
                                               const unsigned tag, const int out_stride, const uint8_t* vp, const unsigned job,
-                                              const size_t warp_off, const int lw, const int lane) {
-    if (b == 0) return chain_items<Q, QC, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 0);
-    return chain_items<Q, QC, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 1);
+                                              const size_t warp_off, const int lw, const int lane, const int wp) {
+    if (b == 0) return chain_items<Q, QC, G, 0>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 0, wp);
+    return chain_items<Q, QC, G, 1>(buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, 1, wp);
 }
 
 // What the roles of a launch share.
@@ -587,7 +598,7 @@ __device__ __forceinline__ const ChainSlot* desc_next(const ChainCtx& x, int slo
 // after every job.
 template <int Q, int G>
 __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
-    const int lane = threadIdx.x & 31, lw = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
     const int h = lane >> 4, l = lane & 15;
     ChainShared* sh = chain_shared();
     uint32_t colp[4];
@@ -603,7 +614,8 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
         // the record in four loads (one round of shared-memory latency instead of a dependent chain of them)
         const uint4* rq = reinterpret_cast<const uint4*>(job_rec(job));
         const uint4 q0 = rq[0], q1 = rq[1], q2 = rq[2], q3 = rq[3];
-        if (q3.z != 0u) break;                                    // stop record
+        if (q3.z & 1u) break;                                     // stop record
+        const int lw = item_slot(wp, (int)(q3.z >> 8));           // this warp's items of the job: lw, lw + 26, ...
         const uint8_t* tile0 = reinterpret_cast<const uint8_t*>(((unsigned long long)q0.y << 32) | q0.x);
         const int rb0 = (int)q0.z, rb1 = (int)q0.w;
         unsigned long long* out = reinterpret_cast<unsigned long long*>(((unsigned long long)q1.y << 32) | q1.x);
@@ -624,7 +636,7 @@ __device__ __forceinline__ void lookup_jobs(const ChainCtx& x) {
             }
             mbar_wait(bar_full(b), (job >> 1) & 1, x.spin_limit, x.status);
             if (sh->abort) return false;
-            carried = chain_items_b<Q, QC, G>(b, buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane);
+            carried = chain_items_b<Q, QC, G>(b, buf, colp, rb0, rb1, out, Y, N, flags, tag, out_stride, vp, job, warp_off, lw, lane, wp);
             if constexpr (Q == 0) {
                 // the part of the buffer that items of this q do not use: given a value here, it is known not to carry one
                 // through the job, which leaves its registers to the look-ups (without this the bodies for q < 4 ran 8 %
@@ -771,6 +783,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
         const int ring = kFinisherWarps + bw;
         const int b = team;
         unsigned job = 0;                                     // jobs of this CTA before the current call
+        unsigned items = 0;                                   // ... and their items, modulo the look-up warps
         for (int c = c_begin; c < c_end; ++c) {
             const ChainSlot* sl = desc_next(x, ring, c, lane);
             const ChainCall* d = &sl->d;
@@ -809,7 +822,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
                         r->flags = d->flags;
                         r->tag = epoch * (unsigned)n_calls + (unsigned)c + 1u;
                         r->last = (seg + 1 == nseg ? 1 : 0) | (d->release ? 2 : 0) | (d->q << 8);
-                        r->stop = 0;
+                        r->stop = (int)((items + (unsigned)seg * (unsigned)(p.rb1 - p.rb0)) % kLookupWarps) << 8;
                         __threadfence_block();
                         mbar_arrive(bar_rec(j));
                     }
@@ -826,6 +839,7 @@ lut_chain_kernel(ChainCtl* ctl, const ChainCall* calls, const int4* parts, unsig
                 }
             }
             job += (unsigned)nseg;
+            items = (items + (unsigned)nseg * (unsigned)(p.rb1 - p.rb0)) % kLookupWarps;
         }
         if ((job & 1u) == (unsigned)team) {
             // the record that ends the look-up warps' loop, handed over like a job (by the team whose turn it is)
