@@ -133,6 +133,12 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), line.strip()))
 
+    def wait_first(self, timeout_s: float = 5.0) -> None:
+        """Returns when the first sample has arrived (nvidia-smi can take a second to start), or after the timeout."""
+        t_end = time.time() + timeout_s
+        while self.proc is not None and not self.rows and time.time() < t_end and self.proc.poll() is None:
+            time.sleep(0.01)
+
     def stop(self, t0: float, t1: float) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -415,6 +421,7 @@ def _secondary(torch, elutq, name, stream, l2_bytes, hbm_peak, tensor_peak, devi
                 sets.append(dup)
         runner = _Runner(torch, elutq, sets, mode, stream)
         sampler = ClockSampler(device_index)
+        sampler.wait_first()
         ms, reps, t0, t1 = runner.timed(10, 5)
         clocks = sampler.stop(t0, t1)
         ms_step = ms / (10 * reps)
@@ -540,6 +547,8 @@ def run_cuda(args) -> None:
 
     # ---- device-resident timing -------------------------------------------------------------
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.wait_first()
     ms, reps, t_wall0, t_wall1 = main.timed(args.steps, args.warmup, barrier)
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     launches = main.launches_per_step * args.steps * reps
@@ -766,7 +775,7 @@ def run_cuda(args) -> None:
         cpu = _cpu_baseline(calls)
 
     if use_chain:
-        launch_desc = ("chained decode entry: elutq_chain_run, one persistent launch per run of equal bit-width "
+        launch_desc = ("chained decode entry: elutq_chain_run, the list of calls in persistent launches "
                        f"({main_launches_per_step(launches, args.steps * reps)} per step), calls ordered as if run one after another")
     elif args.no_graph:
         launch_desc = "stream of C-ABI calls"
