@@ -199,3 +199,32 @@ def test_a_blob_that_changed_under_the_plan_is_refused_before_any_tile_is_read()
     assert elutq.elutq_chain_status(plan) == 0x7C0B
     assert torch.all(Y == 7.0)
     elutq.elutq_forget(buf)
+
+
+def test_list_of_mixed_bit_widths_is_one_launch_and_equals_the_per_q_kernels_bit_for_bit():
+    # G = 128 and q = 1 .. 4 in one list: one launch of the run-time-q instance.  Its look-ups and the order of its
+    # additions are those of the per-q instances (which a list of one bit-width takes), so every output must equal,
+    # bit for bit, what the same call gives as a chain of its own; small and large row counts, one chunk and many.
+    shapes = [(2, 128, 300, 2048), (3, 128, 1000, 4096), (4, 128, 77, 1536), (1, 128, 4096, 512), (2, 128, 6144, 4096),
+              (4, 128, 2048, 1024), (3, 128, 33, 7168), (2, 128, 16, 128)]
+    layers, Xs = _build(shapes, 29, "chain-rtq")
+    packed = [pack_layer(l) for l in layers]
+    xd = [x_dev(x) for x in Xs]
+    Y = [torch.full((1, l.N), float("nan"), dtype=torch.float32, device="cuda") for l in layers]
+    Y1 = [torch.full((1, l.N), float("nan"), dtype=torch.float32, device="cuda") for l in layers]
+    plan = elutq.elutq_chain_plan([(xd[i], packed[i], Y[i], l.N, l.K, elutq.FLAG_OUT_F32) for i, l in enumerate(layers)])
+    torch.cuda.synchronize()
+    n0 = elutq.elutq_launch_count()
+    elutq.elutq_chain_run(plan, len(layers))
+    assert elutq.elutq_launch_count() - n0 == 1
+    assert elutq.elutq_chain_status(plan) == 0
+    for i, l in enumerate(layers):
+        single = elutq.elutq_chain_plan([(xd[i], packed[i], Y1[i], l.N, l.K, elutq.FLAG_OUT_F32)])
+        elutq.elutq_chain_run(single, 1)
+        assert elutq.elutq_chain_status(single) == 0
+        elutq.elutq_chain_forget(single)
+        ref = hlq.matmul(Xs[i], l.planes, l.scales, l.offsets, l.G)
+        y = Y[i].cpu().numpy().astype(np.float64)
+        assert hlq.rel_fro_error(y, ref) <= TOL_F32, (i, shapes[i])
+        assert torch.equal(Y[i].view(torch.int32), Y1[i].view(torch.int32)), (i, shapes[i])
+    elutq.elutq_chain_forget(plan)
