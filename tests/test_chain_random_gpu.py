@@ -22,15 +22,18 @@ TOL_F16 = 1e-3
 DIMS = [128, 256, 512, 1024, 1536, 2048, 4096]          # feature sizes the random layers connect (multiples of 128)
 
 
-def _random_plan(seed):
+LONG_DIMS = [128, 256, 512, 1024, 2048]                 # long lists: small layers (the oracle stays in seconds)
+
+
+def _random_plan(seed, n_lo=4, n_hi=13, dims=DIMS):
     rng = np.random.default_rng(seed)
-    n = int(rng.integers(4, 13))
+    n = int(rng.integers(n_lo, n_hi))
     calls = []
     for i in range(n):
         q = int(rng.integers(1, 5))
         G = int(rng.choice([128, 128, 128, 64, 32]))
-        K = int(rng.choice(DIMS))
-        N = int(rng.choice(DIMS)) - int(rng.choice([0, 0, 0, 3, 17]))        # some ragged row counts
+        K = int(rng.choice(dims))
+        N = int(rng.choice(dims)) - int(rng.choice([0, 0, 0, 3, 17]))        # some ragged row counts
         # with probability 1/3 the call reads the output of an earlier call of matching width
         src = None
         if i > 0 and rng.random() < 0.34:
@@ -45,7 +48,17 @@ def _random_plan(seed):
 
 @pytest.mark.parametrize("seed", list(range(16)))
 def test_random_plans_match_the_oracle_call_by_call(seed):
-    spec = _random_plan(1000 + seed)
+    _check_plan(seed, _random_plan(1000 + seed))
+
+
+@pytest.mark.parametrize("seed", [100, 101, 102, 103])
+def test_long_random_plans_match_the_oracle_call_by_call(seed):
+    # 40 to 64 small calls: the scratch regions are reused many times over (a call waits for the reduction of the call
+    # six before it), the calls' shares wrap around the CTAs several times, and many calls are in flight side by side
+    _check_plan(seed, _random_plan(1000 + seed, 40, 65, LONG_DIMS))
+
+
+def _check_plan(seed, spec):
     layers = [workloads.hlq_layer(seed, f"chain-rand/{seed}/{i}", c["q"], c["G"], c["N"], c["K"], signed_scales=(i % 3 == 0))
               for i, c in enumerate(spec)]
     packed = [pack_layer(l) for l in layers]
