@@ -151,8 +151,8 @@ def test_config1_step_through_the_chain_entry(q):
 
 
 def test_config1_whole_step_as_one_plan():
-    """The benchmark's headline launch configuration: all twelve calls in one plan, which elutq_chain_run turns
-    into one launch per bit-width; run three times (epochs), every output compared in full."""
+    """The benchmark's headline launch configuration: all twelve calls (q = 2, 3, 4) in one plan, which elutq_chain_run
+    runs as one launch; run three times (epochs), every output compared in full."""
     calls = workloads.config1_calls()
     layers = [workloads.hlq_layer(0, c.tag, c.q, c.G, c.N, c.K) for c in calls]
     packed = [pack_layer(l) for l in layers]
