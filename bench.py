@@ -12,8 +12,9 @@ printed by rank 0:
               persistent launch); the same step as separate elutq_lut_gemm calls replayed
               from a CUDA graph is timed beside it (`secondary`).  The working set of a step exceeds
               the L2 capacity
-  e2e         the same metric through elutq_lut_gemm_host: X copied from pinned host memory and Y copied
-              back inside the timed region, every call
+  e2e         the same metric with host buffers, host<->device transfers inside the timed region: M = 1
+              workloads through elutq_chain_run_host (all X in one pinned host arena, fetched by a small kernel;
+              Y stored into a pinned host arena), the others through elutq_lut_gemm_host per call
   roofline    achieved / measured HBM copy bandwidth for the decode kernel
   cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample of the same workload
   secondary   short same-run measurements of the other configurations (70B decode, one 2-bit GEMV
@@ -637,8 +638,8 @@ def run_cuda(args) -> None:
         host_chain_bytes, e2e_how = None, "elutq_lut_gemm_host per call (pinned host X in, Y out), CUDA graph"
         if host_chain is not None:
             host_chain_bytes = (host_chain["h2d"], host_chain["d2h"])
-            e2e_how = ("elutq_chain_run_host: one copy of the pinned host arena of all X in, then the chain's launches, whose "
-                       "calls have their Y in a pinned host arena (the reduction stores straight into host memory), per step")
+            e2e_how = ("elutq_chain_run_host: a fetch kernel reads the pinned host arena of all X across the bus, then the chain's launch, "
+                       "whose calls have their Y in a pinned host arena (the reduction stores straight into host memory), per step")
             e2e_status = elutq.elutq_chain_status(host_chain["plan"], stream=stream)
             if e2e_status:
                 e2e_how += f"; DEVICE STATUS {e2e_status:#x}"

@@ -300,15 +300,21 @@ int elutq_lut_gemm_static(const void* X, const void* packed, void* Y, int M, int
  *   elutq_chain_run_opts    the same with an explicit poll limit for the hand-over waits (0 = default, 2^22);
  *                           a test entry.
  *   elutq_chain_run_host    a run whose activations come from and whose outputs go to HOST memory, with one
- *                           transfer per direction: on `stream`, copies x_bytes from x_host to x_dev, runs the
+ *                           transfer per direction: on `stream`, brings x_bytes from x_host to x_dev, runs the
  *                           plan, copies y_bytes from y_dev to y_host.  x_dev and y_dev are the caller's device
  *                           buffers that the plan's calls point into (typically one arena that holds every
- *                           call's X and one that holds every Y); x_host and y_host should be pinned, otherwise
- *                           the copies are synchronous.  A size of 0 skips that copy: the Y of a call may itself
- *                           name pinned host memory (it is device-accessible under unified addressing), in which
- *                           case the reduction's stores cross the bus while the launch runs and no copy out is
- *                           needed (measured on the twelve 8B calls: 87.5 us per step against 97.1 us with the
- *                           copy; X should NOT be left on the host: every CTA reads it, 1.1 ms).  Returns as elutq_chain_run
+ *                           call's X and one that holds every Y).  Page-locked x_host (16-byte aligned like
+ *                           x_dev, x_bytes a multiple of 16 and at most 8 MiB) is fetched by a small kernel in
+ *                           front of the chain, whose threads read it across the bus, instead of a copy
+ *                           operation, which costs two hand-overs between copy engine and SMs (measured on the
+ *                           twelve 8B calls, 160 KB of activations: 71.5 against 73.8 us per step); any other
+ *                           x_host is copied with cudaMemcpyAsync (synchronous for pageable memory).
+ *                           x_host must stay unchanged until the run has completed.  y_host should be pinned.
+ *                           A size of 0 skips that transfer: the Y of a call may itself name pinned host memory
+ *                           (it is device-accessible under unified addressing), in which case the reduction's
+ *                           stores cross the bus while the launch runs and no copy out is needed (7 us per step
+ *                           less than with the copy; the X of a CALL should not name host memory: every CTA
+ *                           would read it across the bus, 144 us).  Returns as elutq_chain_run
  *                           (ELUTQ_ERR_INVALID_ARG for a null pointer with a non-zero size); the outputs are valid
  *                           on the host when `stream` has been synchronised.  The paper's decode loop keeps
  *                           activations on the device and has no counterpart of this call; it is the end-to-end

@@ -152,6 +152,22 @@ def test_chain_with_host_buffers_moves_one_arena_per_direction():
     for i, l in enumerate(layers):
         a, b = int(y_off[i]), int(y_off[i]) + l.N
         assert torch.equal(y_host2[a:b].view(torch.int16), y_host[a:b].view(torch.int16)), shapes[i]
+    # Pinned activations are fetched by a kernel that reads them across the bus, pageable ones go through a copy: the
+    # same bits either way, also when the run is repeated with other activations and between runs that fetch nothing
+    x_alt = (x_host.float() * 0.5).half()
+    for rep, xs in enumerate((x_alt, x_host)):
+        for pinned in (True, False):
+            src = xs.clone().pin_memory() if pinned else xs.clone()
+            y_host2.fill_(float("nan"))
+            elutq.elutq_chain_run_host(plan2, len(calls), x_dev, src)
+            assert elutq.elutq_chain_status(plan2) == 0
+            assert torch.equal(x_dev.cpu().view(torch.int16), xs.view(torch.int16))
+            elutq.elutq_chain_run(plan2, len(calls))                 # X resident: nothing fetched, same outputs
+            assert elutq.elutq_chain_status(plan2) == 0
+            if rep == 1:
+                for i, l in enumerate(layers):
+                    a, b = int(y_off[i]), int(y_off[i]) + l.N
+                    assert torch.equal(y_host2[a:b].view(torch.int16), y_host[a:b].view(torch.int16)), (shapes[i], pinned)
     elutq.elutq_chain_forget(plan)
     elutq.elutq_chain_forget(plan2)
 
