@@ -345,6 +345,14 @@ int elutq_chain_status(const void* plan, void* stream, int* status);
  * elutq_chain_run returns ELUTQ_ERR_SHAPE for a buffer that this process has not planned.  Call this before
  * freeing a plan buffer. */
 int elutq_chain_forget(const void* plan);
+/* Host logic of elutq_chain_plan for ONE call, without any CUDA call (for tests and for sizing questions): how a call
+ * of shape (N, K) is cut over the n_ctas_max CTAs of a launch.  shares: int [n_ctas_max][4], per CTA (first row
+ * block, end row block, first chunk, chunks | chunk group << 16), zeros for a CTA without a share; row blocks are 16
+ * rows, chunks 512 columns; the shares go to CTAs cta_first, cta_first + 1, ... modulo n_ctas_max, as in a plan, where
+ * cta_first is the sum of the earlier calls' CTA counts.  independent != 0: the call neither waits for the call before
+ * it nor is waited for by the call after it (a small such call takes fewer CTAs).  partition: int [4] = chunks per
+ * CTA, row ranges, chunk groups, CTAs with a share.  ELUTQ_ERR_UNSUPPORTED: more chunk groups than CTAs. */
+int elutq_chain_shares(int N, int K, int n_ctas_max, int cta_first, int independent, int* shares, int* partition);
 
 /*
  * Algorithm 1 (Section 4.2): alternating optimisation of the HLQ parameters, the offline step that

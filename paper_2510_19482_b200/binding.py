@@ -63,6 +63,7 @@ _SIGNATURES = {
     "elutq_chain_run_host": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_size_t, c_void_p]),
     "elutq_chain_status": (c_int, [c_void_p, c_void_p, ctypes.POINTER(c_int)]),
     "elutq_chain_forget": (c_int, [c_void_p]),
+    "elutq_chain_shares": (c_int, [c_int, c_int, c_int, c_int, c_int, ctypes.POINTER(c_int), ctypes.POINTER(c_int)]),
     "elutq_device_status": (c_int, [c_void_p, ctypes.POINTER(c_int)]),
     "elutq_launch_count": (c_ulonglong, []),
     "elutq_release_scratch": (c_int, []),
@@ -272,6 +273,16 @@ def elutq_chain_status(plan, stream=None) -> int:
 
 def elutq_chain_forget(plan) -> None:
     _check(lib().elutq_chain_forget(_ptr(plan)), "elutq_chain_forget")
+
+
+def elutq_chain_shares(N: int, K: int, n_ctas_max: int, cta_first: int = 0, independent: bool = True):
+    """(shares, partition): shares[cta] = (first row block, end row block, first chunk, chunks, chunk group);
+    partition = (chunks per CTA, row ranges, chunk groups, CTAs with a share).  Host logic only."""
+    raw = (c_int * (4 * n_ctas_max))()
+    part = (c_int * 4)()
+    _check(lib().elutq_chain_shares(N, K, n_ctas_max, cta_first, 1 if independent else 0, raw, part), "elutq_chain_shares")
+    shares = [(raw[4 * i], raw[4 * i + 1], raw[4 * i + 2], raw[4 * i + 3] & 0xffff, raw[4 * i + 3] >> 16) for i in range(n_ctas_max)]
+    return shares, tuple(part)
 
 
 def elutq_reserve(M: int, N: int, K: int, stream=None) -> None:

@@ -949,6 +949,48 @@ ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls, int sms) {
     return L;
 }
 
+// A call's partition over the CTAs of a launch and every CTA's share of it (host logic only, no CUDA call).
+// n_rb row blocks x n_kc chunks are cut into `groups` groups of cpc consecutive chunks times R row ranges, one
+// share (a row-block range of one chunk group) per CTA; the shares go to CTAs cta_first, cta_first + 1, ... modulo
+// the CTA count.  share[cta] = (first row block, end row block, first chunk, chunks | group << 16); zeros: no share.
+// A job with fewer items than look-up warps leaves warps idle while it lasts about as long (an item is mostly a load
+// round trip), so a small layer spread over every SM costs every SM a full job cycle.  A small call that is
+// independent of its neighbours in the list takes fewer CTAs instead - two rounds of items for every look-up warp of
+// a CTA - and consecutive calls start on different CTAs: such calls then run side by side on different SMs.
+// (Measured, 8B shapes: chains of attention-output layers 2.16 -> 1.67 us per call at q = 2, 3.50 -> 2.40 at q = 4;
+// the 12-call step 63.0 -> 59.2 us; a chain in which every call reads the output of the one before is fastest spread
+// over every SM.)
+struct CallPartition {
+    int cpc, ranges, groups, n_ctas;
+};
+bool chain_shares(int n_rb, int n_kc, int sms, int cta_first, bool independent, CallPartition* part, int4* share) {
+    int cpc = 1, R = 1;
+    plan_gemv_partition(n_rb, n_kc, sms, false, &cpc, &R);
+    if (cpc == 1 && independent) {
+        const int fill = (n_rb + 2 * kLookupWarps - 1) / (2 * kLookupWarps);
+        if (R > fill) R = fill;
+    }
+    part->cpc = cpc; part->ranges = R;
+    part->groups = (n_kc + cpc - 1) / cpc;
+    part->n_ctas = part->groups * R;
+    if (part->n_ctas > sms || part->n_ctas <= 0) return false;
+    const int rb_q = n_rb / R, rb_r = n_rb % R;
+    for (int cta = 0; cta < sms; ++cta) {
+        int4 v = make_int4(0, 0, 0, 0);
+        const int b = (cta - cta_first % sms + sms) % sms;
+        if (b < part->n_ctas) {
+            const int grp = b / R, range = b - grp * R;
+            v.x = range * rb_q + (range < rb_r ? range : rb_r);
+            v.y = v.x + rb_q + (range < rb_r ? 1 : 0);
+            v.z = grp * cpc;
+            const int nseg = (cpc < n_kc - v.z) ? cpc : n_kc - v.z;
+            v.w = nseg | (grp << 16);
+        }
+        share[cta] = v;
+    }
+    return true;
+}
+
 int check_call(const elutq_gemv_call& c) {
     if (!c.X || !c.packed || !c.Y) return ELUTQ_ERR_INVALID_ARG;
     if (c.N <= 0 || c.K <= 0) return ELUTQ_ERR_INVALID_ARG;
@@ -1094,40 +1136,15 @@ int elutq_chain_plan(const elutq_gemv_call* calls, int n_calls, void* plan, size
         ChainCall& d = dc[i];
         const int q = d.q, G = d.G;
         const Geo g = make_geo(q, G, c.N, c.K);
-        int cpc = 1, R = 1;
-        plan_gemv_partition(g.n_rb, g.n_kc, sms, false, &cpc, &R);
-        // A job with fewer items than look-up warps leaves warps idle while it lasts about as long (an item is mostly
-        // a load round trip), so a small layer spread over every SM costs every SM a full job cycle.  A small call
-        // that neither waits for the call before it nor is waited for by the call after it takes fewer CTAs instead
-        // - two rounds of items for every look-up warp of a CTA - and consecutive calls start on different CTAs
-        // (cta_first below): such calls then run side by side on different SMs.  (Measured, 8B shapes: chains of
-        // attention-output layers 2.16 -> 1.67 us per call at q = 2, 3.50 -> 2.40 at q = 4; the 12-call step 63.0 ->
-        // 59.2 us; a chain in which every call reads the output of the one before is fastest spread over every SM.)
+        // a call that neither waits for the call before it nor is waited for by the call after it may take fewer CTAs
         const bool waits = d.dep_first <= d.dep_last && d.dep_last == i - 1;
         const bool waited_for = i + 1 < n_calls && dc[i + 1].dep_first <= dc[i + 1].dep_last && dc[i + 1].dep_last == i;
-        if (cpc == 1 && !waits && !waited_for) {
-            const int fill = (g.n_rb + 2 * kLookupWarps - 1) / (2 * kLookupWarps);
-            if (R > fill) R = fill;
-        }
-        d.cpc = cpc; d.ranges = R; d.rb_q = g.n_rb / R; d.rb_r = g.n_rb % R;
-        d.groups = (g.n_kc + cpc - 1) / cpc;
-        d.n_ctas = d.groups * R;
-        if (d.n_ctas > sms) return ELUTQ_ERR_UNSUPPORTED;
-        // every CTA's share of the call: row-block range, first chunk, chunks, chunk group
+        CallPartition cp;
         int4* pt = reinterpret_cast<int4*>(host.data() + L.parts_off) + (size_t)i * sms;
-        for (int cta = 0; cta < sms; ++cta) {
-            int4 v = make_int4(0, 0, 0, 0);
-            const int b = (cta - cta_first + sms) % sms;      // the call's shares go to CTAs cta_first, cta_first + 1, ... (mod)
-            if (b < d.n_ctas) {
-                const int grp = b / R, range = b - grp * R;
-                v.x = range * d.rb_q + (range < d.rb_r ? range : d.rb_r);
-                v.y = v.x + d.rb_q + (range < d.rb_r ? 1 : 0);
-                v.z = grp * cpc;
-                const int nseg = (cpc < g.n_kc - v.z) ? cpc : g.n_kc - v.z;
-                v.w = nseg | (grp << 16);
-            }
-            pt[cta] = v;
-        }
+        if (!chain_shares(g.n_rb, g.n_kc, sms, cta_first, !waits && !waited_for, &cp, pt)) return ELUTQ_ERR_UNSUPPORTED;
+        d.cpc = cp.cpc; d.ranges = cp.ranges; d.rb_q = g.n_rb / cp.ranges; d.rb_r = g.n_rb % cp.ranges;
+        d.groups = cp.groups;
+        d.n_ctas = cp.n_ctas;
         cta_first = (cta_first + d.n_ctas) % sms;
         d.guard_call = i >= L.regions ? i - L.regions : -1;
         d.guard_target = d.guard_call >= 0 ? dc[d.guard_call].done_target : 0u;
@@ -1240,6 +1257,19 @@ int elutq_chain_status(const void* plan, void* stream, int* status) {
     return ELUTQ_OK;
 }
 
+
+int elutq_chain_shares(int N, int K, int n_ctas_max, int cta_first, int independent, int* shares, int* partition) {
+    if (N <= 0 || K <= 0 || n_ctas_max <= 0 || n_ctas_max > 1024 || cta_first < 0 || !shares || !partition) return ELUTQ_ERR_INVALID_ARG;
+    const int n_rb = (N + kTileRows - 1) / kTileRows, n_kc = (K + kChunkK - 1) / kChunkK;
+    CallPartition cp;
+    std::vector<int4> sh((size_t)n_ctas_max);
+    if (!chain_shares(n_rb, n_kc, n_ctas_max, cta_first, independent != 0, &cp, sh.data())) return ELUTQ_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_ctas_max; ++i) {
+        shares[4 * i] = sh[i].x; shares[4 * i + 1] = sh[i].y; shares[4 * i + 2] = sh[i].z; shares[4 * i + 3] = sh[i].w;
+    }
+    partition[0] = cp.cpc; partition[1] = cp.ranges; partition[2] = cp.groups; partition[3] = cp.n_ctas;
+    return ELUTQ_OK;
+}
 
 int elutq_chain_forget(const void* plan) {
     if (!plan) return ELUTQ_ERR_INVALID_ARG;
