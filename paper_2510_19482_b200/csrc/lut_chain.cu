@@ -44,8 +44,8 @@ namespace {
 
 constexpr unsigned kChainMagic = 0x4E494843u;
 constexpr int kChainRegions = 6;              // scratch regions for the tagged partial sums, used round-robin: at least
-constexpr int kChainRegionsMax = 12;          // this many, more (up to the maximum) while they stay within the budget
-constexpr size_t kChainScratchBudget = 12u << 20;
+constexpr int kChainRegionsMax = 12;          // this many, more (up to the maximum) while all of them fit kChainScratchBytes
+constexpr size_t kChainScratchBytes = 12u << 20;
 constexpr int kDescSlots = 4;
 constexpr int kLookupWarps = 26;              // (22 or 18 look-up warps with 72 / 80 registers each measured slower)
 constexpr int kBuilderWarps = 4;
@@ -943,7 +943,7 @@ ChainLayout chain_layout(const elutq_gemv_call* calls, int n_calls, int sms) {
     L.slots_off = L.parts_off + round_up((size_t)n_calls * sms * sizeof(int4), 256);
     // Lists of small calls keep more calls in flight (they run side by side on different SMs): more regions, measured
     // on chains of the 8B attention-output layer 1.67 -> 1.54 us per call with ten instead of six.
-    size_t regions = kChainScratchBudget / L.region_bytes;
+    size_t regions = kChainScratchBytes / L.region_bytes;
     L.regions = (int)(regions < (size_t)kChainRegions ? (size_t)kChainRegions : regions > (size_t)kChainRegionsMax ? (size_t)kChainRegionsMax : regions);
     L.total = L.slots_off + (size_t)L.regions * L.region_bytes;
     return L;

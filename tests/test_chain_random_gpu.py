@@ -54,7 +54,7 @@ def test_random_plans_match_the_oracle_call_by_call(seed):
 @pytest.mark.parametrize("seed", [100, 101, 102, 103])
 def test_long_random_plans_match_the_oracle_call_by_call(seed):
     # 40 to 64 small calls: the scratch regions are reused many times over (a call waits for the reduction of the call
-    # six before it), the calls' shares wrap around the CTAs several times, and many calls are in flight side by side
+    # that used its region last, six to twelve calls before it), the calls' shares wrap around the CTAs several times, and many calls are in flight side by side
     _check_plan(seed, _random_plan(1000 + seed, 40, 65, LONG_DIMS))
 
 
